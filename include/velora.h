@@ -1,0 +1,165 @@
+/*
+ * velora.h -- C-ABI of the B200 (sm_100a) VeLoRA linear-layer library.
+ *
+ * VeLoRA (arxiv 2405.17991) replaces the input X[N, D] that a linear layer
+ * saves for its backward pass by one scalar per sub-token: every token is cut
+ * into M = ceil(D / Dsub) contiguous sub-tokens of length Dsub and each is
+ * projected onto one fixed unit vector v[Dsub] (Section 3.1).  The backward
+ * pass rebuilds a coarse input Xhat = Z (x) v for the weight gradient
+ * (Algorithm 1).
+ *
+ * Naming.  The paper calls the sub-token LENGTH "M"; this header calls it
+ * Dsub and uses M for the NUMBER of sub-tokens per token.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library
+ *     never allocates or frees device memory and keeps no state between calls
+ *     (only a per-process cache of immutable launch attributes).  Scratch is a
+ *     caller-provided device workspace sized by velora_workspace_bytes().
+ *   - Matrices are row-major with an explicit leading dimension counted in
+ *     ELEMENTS.  W is [O, D] (nn.Linear convention): Y = X W^T, dX = dY W,
+ *     dW = dY^T Xhat.  The listing in Algorithm 1 is only consistent with
+ *     this layout.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Work is enqueued asynchronously; only velora_init_v synchronises.
+ *   - Return value: a velora_status.  Arguments are validated on the host
+ *     before anything is launched; on a non-zero status no output is written
+ *     (VELORA_ERR_CUDA and VELORA_ERR_TIMEOUT excepted, which report a failure
+ *     of an already enqueued launch).  Nothing throws, aborts or prints.
+ *   - When Dsub does not divide D the last sub-token is the remaining
+ *     D - (M-1)*Dsub entries followed by zeros (the paper's group() is a
+ *     reshape and is silent on this case); outputs of width D are written on
+ *     their first D columns only.
+ *   - N == 0 is a successful no-op (velora_init_v: VELORA_ERR_DEGENERATE_V).
+ *   - Vector (128-bit) kernels are used when base pointers are 16-byte aligned,
+ *     leading dimensions are multiples of 16 bytes and Dsub is a multiple of 8;
+ *     otherwise the element-wise kernels run (same results, lower speed).  The
+ *     tensor-core GEMMs need 16-byte aligned bf16 rows; other cases run on the
+ *     CUDA-core GEMM.
+ */
+#ifndef VELORA_H
+#define VELORA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    VELORA_OK = 0,
+    VELORA_ERR_INVALID_ARG = 1,   /* null pointer, negative size, ld < width, Dsub out of range */
+    VELORA_ERR_UNSUPPORTED = 2,   /* dtype combination or size outside what the kernels cover  */
+    VELORA_ERR_ALIGNMENT = 3,     /* pointer not aligned to its element size                   */
+    VELORA_ERR_WORKSPACE = 4,     /* workspace missing or smaller than velora_workspace_bytes  */
+    VELORA_ERR_DEGENERATE_V = 5,  /* the sub-token sum has zero or non-finite length           */
+    VELORA_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired (reported by status)   */
+    VELORA_ERR_CUDA = 7           /* a CUDA runtime call or launch failed                      */
+} velora_status;
+
+typedef enum { VELORA_F32 = 0, VELORA_BF16 = 1 } velora_dtype;
+
+/* How velora_weight_grad forms dW. */
+typedef enum {
+    VELORA_WG_FACTORED = 0,  /* P = dY^T Z on tensor cores, dW = P (x) v in the epilogue; Xhat never exists */
+    VELORA_WG_EXPLICIT = 1   /* Xhat = reconstruct(Z, v) into the workspace, then the dense GEMM dY^T Xhat    */
+} velora_wg_mode;
+
+typedef enum {
+    VELORA_OP_INIT_V = 0,
+    VELORA_OP_WEIGHT_GRAD_FACTORED = 1,
+    VELORA_OP_WEIGHT_GRAD_EXPLICIT = 2,
+    VELORA_OP_LINEAR_FORWARD = 3,
+    VELORA_OP_LINEAR_BACKWARD_FACTORED = 4,
+    VELORA_OP_LINEAR_BACKWARD_EXPLICIT = 5
+} velora_op;
+
+#define VELORA_MAX_DSUB 1024
+
+/* Library version, major*10000 + minor*100 + patch. */
+int velora_version(void);
+
+/* Static, human-readable name of a status code. */
+const char* velora_status_string(int status);
+
+/*
+ * Bytes of device workspace the given entry point needs for these sizes
+ * (0 if it needs none).  Independent of pointer values; deterministic.
+ */
+size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub);
+
+/*
+ * Initialise the projection vector from a batch (Section 3.2, "Cheap
+ * initialisation strategies": the average of the first batch's sub-tokens;
+ * Section 3.1: v has unit length):
+ *     s[j] = sum_n sum_m X[n, m*Dsub + j],   v = s / ||s||_2      (fp32, v[Dsub])
+ * X: [N, D], x_dtype bf16 or f32, leading dimension ldx.  The sum over tokens
+ * uses a fixed order, so results are run-to-run identical.
+ * ws: device workspace of velora_workspace_bytes(VELORA_OP_INIT_V, ...) bytes.
+ * Synchronises `stream` once to read back whether the sum is degenerate;
+ * returns VELORA_ERR_DEGENERATE_V and leaves v untouched if ||s|| is zero or
+ * not finite.
+ */
+int velora_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                  float* v, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * compress (Section 3.1, Eq. 1):  Z[n, m] = sum_j X[n, m*Dsub + j] * v[j].
+ * X: [N, D] bf16 or f32.  v: fp32 [Dsub].  Z: [N, M] f32 or bf16, ldz >= M.
+ * Products and sums are formed in fp32.
+ */
+int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                    const float* v, void* Z, int z_dtype, int64_t ldz, void* stream);
+
+/*
+ * reconstruct + ungroup (Section 3.1, Eq. 2):  Xhat[n, m*Dsub + j] = Z[n, m] * v[j].
+ * Z: [N, M] f32 or bf16.  Xhat: [N, D] bf16 or f32 (rounded to nearest even).
+ */
+int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
+                       const float* v, void* Xhat, int x_dtype, int64_t ldxhat, void* stream);
+
+/*
+ * Weight gradient of Algorithm 1's backward with the reconstructed input:
+ *     dW[o, d] = beta * dW[o, d] + sum_n dY[n, o] * Xhat[n, d],  Xhat = Z (x) v
+ * dY: [N, O] bf16 or f32.  Z: [N, M] f32 or bf16.  dW: [O, D] bf16 or f32.
+ * beta is 0 (overwrite) or 1 (accumulate into dW).
+ * mode VELORA_WG_FACTORED uses dW[o, m*Dsub+j] = (dY^T Z)[o, m] * v[j]
+ * (the Dsub = D case is the paper's g v v^T, Section 3.2); VELORA_WG_EXPLICIT
+ * materialises Xhat in the workspace and multiplies -- kept as a cross-check.
+ * ws: velora_workspace_bytes(VELORA_OP_WEIGHT_GRAD_{FACTORED,EXPLICIT}, N, D, O, Dsub).
+ */
+int velora_weight_grad(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                       const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                       void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Forward of the VeLoRA linear (Algorithm 1, forward):
+ *     Y[N, O] = X W^T      and      Z = compress(X, v)
+ * `dtype` is the storage type of X, W and Y (bf16: tensor cores with fp32
+ * accumulation; f32: CUDA cores).  Z as in velora_compress.  X itself need not
+ * be kept by the caller afterwards: (Z, W, v) is all the backward needs.
+ * ws: velora_workspace_bytes(VELORA_OP_LINEAR_FORWARD, ...) bytes (may be 0 / NULL).
+ */
+int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
+                          void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
+                          int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Backward of the VeLoRA linear (Algorithm 1, backward):
+ *     dX[N, D] = dY W                  (exact; skipped when dX == NULL)
+ *     dW[O, D] as velora_weight_grad   (skipped when dW == NULL)
+ * `dtype` is the storage type of dY, W and dX.
+ */
+int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t ldw,
+                           const void* Z, int z_dtype, int64_t ldz, const float* v,
+                           void* dX, int64_t lddx, void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
+                           int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
+                           void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VELORA_H */

@@ -1,0 +1,231 @@
+"""ctypes binding of libvelora.so: argument marshalling only.
+
+Each function has the name and meaning of the C entry point it wraps
+(``include/velora.h``); tensors are torch CUDA tensors whose device memory,
+row pitch and current stream are handed to the library as plain pointers and
+integers.  Every step of the path runs inside the library's kernels; there is
+no fallback: a missing library or a non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvelora.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_DEGENERATE_V, ERR_TIMEOUT, ERR_CUDA = range(8)
+F32, BF16 = 0, 1
+WG_FACTORED, WG_EXPLICIT = 0, 1
+(OP_INIT_V, OP_WEIGHT_GRAD_FACTORED, OP_WEIGHT_GRAD_EXPLICIT, OP_LINEAR_FORWARD,
+ OP_LINEAR_BACKWARD_FACTORED, OP_LINEAR_BACKWARD_EXPLICIT) = range(6)
+
+_p, _i64, _int, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+
+SIGNATURES = {
+    "velora_version": (_int, []),
+    "velora_status_string": (ctypes.c_char_p, [_int]),
+    "velora_workspace_bytes": (_sz, [_int, _i64, _i64, _i64, _int]),
+    "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
+    "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
+    "velora_reconstruct": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
+    "velora_weight_grad": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _p, _i64, _int,
+                                  _p, _int, _i64, _int, _int, _p, _sz, _p]),
+    "velora_linear_forward": (_int, [_p, _i64, _p, _i64, _p, _p, _i64, _p, _int, _i64,
+                                     _int, _i64, _i64, _i64, _int, _p, _sz, _p]),
+    "velora_linear_backward": (_int, [_p, _i64, _p, _i64, _p, _int, _i64, _p, _p, _i64, _p, _int, _i64, _int, _int,
+                                      _int, _i64, _i64, _i64, _int, _p, _sz, _p]),
+}
+
+
+class VeloraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().velora_status_string(status).decode()
+        super().__init__("%s: status %d (%s)" % (where, status, msg))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libvelora.so is missing at %s: build it with `python -m paper_2405_17991_b200.build` "
+                "(nvcc, sm_100a). There is no CPU or PyTorch fallback." % LIB_PATH)
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("unsupported dtype %s (float32 or bfloat16)" % t.dtype)
+
+
+def _mat(t: torch.Tensor, name: str):
+    if t.ndim != 2 or not t.is_cuda:
+        raise ValueError("%s must be a 2-d CUDA tensor" % name)
+    if t.shape[1] > 1 and t.stride(1) != 1:
+        raise ValueError("%s must have contiguous rows" % name)
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+    return ctypes.c_void_p(t.data_ptr()), int(ld)
+
+
+def _vec(v: torch.Tensor):
+    if v.ndim != 1 or v.dtype != torch.float32 or not v.is_cuda or not v.is_contiguous():
+        raise ValueError("v must be a contiguous 1-d float32 CUDA tensor")
+    return ctypes.c_void_p(v.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ws(ws: Optional[torch.Tensor], need: int, device) -> torch.Tensor:
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+    return ws
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise VeloraError(status, where)
+
+
+def num_subtokens(D: int, Dsub: int) -> int:
+    return -(-D // Dsub)
+
+
+def velora_version() -> int:
+    return lib().velora_version()
+
+
+def velora_status_string(status: int) -> str:
+    return lib().velora_status_string(status).decode()
+
+
+def velora_workspace_bytes(op: int, N: int, D: int, O: int, Dsub: int) -> int:
+    return int(lib().velora_workspace_bytes(op, N, D, O, Dsub))
+
+
+def velora_init_v(X: torch.Tensor, Dsub: int, v: Optional[torch.Tensor] = None,
+                  ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    xp, ldx = _mat(X, "X")
+    N, D = X.shape
+    if v is None:
+        v = torch.empty(Dsub, dtype=torch.float32, device=X.device)
+    ws = _ws(ws, velora_workspace_bytes(OP_INIT_V, N, D, 1, Dsub), X.device)
+    rc = lib().velora_init_v(xp, _dt(X), N, D, ldx, Dsub, _vec(v), ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                             _stream(stream))
+    _check(rc, "velora_init_v")
+    return v
+
+
+def velora_compress(X: torch.Tensor, v: torch.Tensor, Z: Optional[torch.Tensor] = None,
+                    z_dtype=torch.float32, stream=None) -> torch.Tensor:
+    xp, ldx = _mat(X, "X")
+    N, D = X.shape
+    Dsub = v.shape[0]
+    if Z is None:
+        Z = torch.empty((N, num_subtokens(D, Dsub)), dtype=z_dtype, device=X.device)
+    zp, ldz = _mat(Z, "Z")
+    rc = lib().velora_compress(xp, _dt(X), N, D, ldx, Dsub, _vec(v), zp, _dt(Z), ldz, _stream(stream))
+    _check(rc, "velora_compress")
+    return Z
+
+
+def velora_reconstruct(Z: torch.Tensor, v: torch.Tensor, D: int, Xhat: Optional[torch.Tensor] = None,
+                       x_dtype=torch.bfloat16, stream=None) -> torch.Tensor:
+    zp, ldz = _mat(Z, "Z")
+    N = Z.shape[0]
+    Dsub = v.shape[0]
+    if Xhat is None:
+        Xhat = torch.empty((N, D), dtype=x_dtype, device=Z.device)
+    xp, ldx = _mat(Xhat, "Xhat")
+    rc = lib().velora_reconstruct(zp, _dt(Z), ldz, N, D, Dsub, _vec(v), xp, _dt(Xhat), ldx, _stream(stream))
+    _check(rc, "velora_reconstruct")
+    return Xhat
+
+
+def velora_weight_grad(dY: torch.Tensor, Z: torch.Tensor, v: torch.Tensor, D: int,
+                       dW: Optional[torch.Tensor] = None, dw_dtype=None, beta: int = 0, mode: int = WG_FACTORED,
+                       ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    yp, lddy = _mat(dY, "dY")
+    zp, ldz = _mat(Z, "Z")
+    N, O = dY.shape
+    Dsub = v.shape[0]
+    if dW is None:
+        dW = torch.empty((O, D), dtype=dw_dtype or dY.dtype, device=dY.device)
+    wp, lddw = _mat(dW, "dW")
+    op = OP_WEIGHT_GRAD_FACTORED if mode == WG_FACTORED else OP_WEIGHT_GRAD_EXPLICIT
+    ws = _ws(ws, velora_workspace_bytes(op, N, D, O, Dsub), dY.device)
+    rc = lib().velora_weight_grad(yp, _dt(dY), N, O, lddy, zp, _dt(Z), ldz, _vec(v), D, Dsub,
+                                  wp, _dt(dW), lddw, beta, mode, ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                  _stream(stream))
+    _check(rc, "velora_weight_grad")
+    return dW
+
+
+def velora_linear_forward(X: torch.Tensor, W: torch.Tensor, v: torch.Tensor,
+                          Y: Optional[torch.Tensor] = None, Z: Optional[torch.Tensor] = None,
+                          z_dtype=torch.float32, ws: Optional[torch.Tensor] = None, stream=None):
+    xp, ldx = _mat(X, "X")
+    wp, ldw = _mat(W, "W")
+    N, D = X.shape
+    O = W.shape[0]
+    Dsub = v.shape[0]
+    if W.shape[1] != D or W.dtype != X.dtype:
+        raise ValueError("W must be [O, D] with X's dtype")
+    if Y is None:
+        Y = torch.empty((N, O), dtype=X.dtype, device=X.device)
+    if Z is None:
+        Z = torch.empty((N, num_subtokens(D, Dsub)), dtype=z_dtype, device=X.device)
+    yp, ldy = _mat(Y, "Y")
+    zp, ldz = _mat(Z, "Z")
+    ws = _ws(ws, velora_workspace_bytes(OP_LINEAR_FORWARD, N, D, O, Dsub), X.device)
+    rc = lib().velora_linear_forward(xp, ldx, wp, ldw, _vec(v), yp, ldy, zp, _dt(Z), ldz,
+                                     _dt(X), N, D, O, Dsub, ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                     _stream(stream))
+    _check(rc, "velora_linear_forward")
+    return Y, Z
+
+
+def velora_linear_backward(dY: torch.Tensor, W: torch.Tensor, Z: torch.Tensor, v: torch.Tensor,
+                           dX: Optional[torch.Tensor] = None, dW: Optional[torch.Tensor] = None,
+                           need_dX: bool = True, need_dW: bool = True, dw_dtype=None, beta: int = 0,
+                           mode: int = WG_FACTORED, ws: Optional[torch.Tensor] = None, stream=None):
+    yp, lddy = _mat(dY, "dY")
+    wp, ldw = _mat(W, "W")
+    zp, ldz = _mat(Z, "Z")
+    N, O = dY.shape
+    D = W.shape[1]
+    Dsub = v.shape[0]
+    if need_dX and dX is None:
+        dX = torch.empty((N, D), dtype=dY.dtype, device=dY.device)
+    if need_dW and dW is None:
+        dW = torch.empty((O, D), dtype=dw_dtype or dY.dtype, device=dY.device)
+    xp, lddx = _mat(dX, "dX") if need_dX else (ctypes.c_void_p(0), D)
+    gp, lddw = _mat(dW, "dW") if need_dW else (ctypes.c_void_p(0), D)
+    op = OP_LINEAR_BACKWARD_FACTORED if mode == WG_FACTORED else OP_LINEAR_BACKWARD_EXPLICIT
+    ws = _ws(ws, velora_workspace_bytes(op, N, D, O, Dsub), dY.device)
+    rc = lib().velora_linear_backward(yp, lddy, wp, ldw, zp, _dt(Z), ldz, _vec(v), xp, lddx,
+                                      gp, _dt(dW) if need_dW else _dt(dY), lddw, beta, mode,
+                                      _dt(dY), N, D, O, Dsub, ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                      _stream(stream))
+    _check(rc, "velora_linear_backward")
+    return dX, dW

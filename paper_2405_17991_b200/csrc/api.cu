@@ -1,0 +1,269 @@
+// C-ABI entry points of the VeLoRA library: host-side validation and routing.
+// Every argument check happens here, before any launch.
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+namespace velora {
+
+int device_info(DeviceInfo* out)
+{
+    static DeviceInfo cache[64];
+    static bool have[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return VELORA_ERR_UNSUPPORTED;
+    if (!have[dev]) {
+        DeviceInfo di;
+        if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return VELORA_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&di.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return VELORA_ERR_CUDA;
+        cache[dev] = di;
+        have[dev] = true;
+    }
+    *out = cache[dev];
+    return VELORA_OK;
+}
+
+namespace {
+
+bool elem_aligned(const void* p, int dt)
+{
+    return (reinterpret_cast<uintptr_t>(p) % dtype_size(dt)) == 0;
+}
+
+int check_shape(int64_t N, int64_t D, int Dsub)
+{
+    if (N < 0 || D < 1 || Dsub < 1 || Dsub > D) return VELORA_ERR_INVALID_ARG;
+    if (Dsub > VELORA_MAX_DSUB) return VELORA_ERR_UNSUPPORTED;
+    if (D > (1 << 30) || N > (static_cast<int64_t>(1) << 40)) return VELORA_ERR_UNSUPPORTED;
+    return VELORA_OK;
+}
+
+int64_t num_subtokens(int64_t D, int Dsub) { return ceil_div64(D, Dsub); }
+
+int64_t round_up8(int64_t x) { return (x + 7) / 8 * 8; }
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t xhat_bytes(int64_t N, int64_t D) { return align256(static_cast<size_t>(N) * round_up8(D) * 4); }
+
+size_t factored_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
+{
+    const size_t simt = align256(static_cast<size_t>(O) * num_subtokens(D, Dsub) * sizeof(float));
+    const size_t tc = weight_grad_tc_workspace_bytes(N, D, O, Dsub);
+    return kStatusBytes + (simt > tc ? simt : tc);
+}
+
+// ---- weight gradient routing ----
+int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                     const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                     void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
+                     void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    const int64_t M = num_subtokens(D, Dsub);
+    if (mode == VELORA_WG_FACTORED) {
+        if (ws_bytes < factored_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
+        char* body = static_cast<char*>(ws) + kStatusBytes;
+        int rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
+                                       dW, dw_dtype, lddw, beta, body, ws_bytes - kStatusBytes, stream);
+        if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+        // CUDA-core route: P[O, M] = dY^T Z, then the outer-product expansion.
+        float* P = reinterpret_cast<float*>(body);
+        rc = launch_gemm_simt(dY, dy_dtype, 1, lddy, Z, z_dtype, 1, ldz, P, VELORA_F32, M, 0, O, M, N, stream);
+        if (rc != VELORA_OK) return rc;
+        return launch_expand_p(P, M, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
+    }
+    // Explicit: Xhat into the workspace in dY's storage type, then dW = dY^T Xhat.
+    if (ws_bytes < xhat_bytes(N, D)) return VELORA_ERR_WORKSPACE;
+    const int64_t ldxh = round_up8(D);
+    int rc = launch_reconstruct(Z, z_dtype, ldz, N, D, Dsub, v, ws, dy_dtype, ldxh, stream);
+    if (rc != VELORA_OK) return rc;
+    rc = launch_gemm_tc(GEMM_TN_MN_MN, dY, lddy, ws, ldxh, dW, dw_dtype, lddw, beta, O, D, N, dy_dtype, stream);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    return launch_gemm_simt(dY, dy_dtype, 1, lddy, ws, dy_dtype, 1, ldxh, dW, dw_dtype, lddw, beta, O, D, N, stream);
+}
+
+int check_weight_grad_args(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                           const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                           void* dW, int dw_dtype, int64_t lddw, int beta, int mode, void* ws)
+{
+    if (!dY || !Z || !v || !dW) return VELORA_ERR_INVALID_ARG;
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(dy_dtype) || !valid_dtype(z_dtype) || !valid_dtype(dw_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (lddy < O || ldz < num_subtokens(D, Dsub) || lddw < D) return VELORA_ERR_INVALID_ARG;
+    if ((beta != 0 && beta != 1) || (mode != VELORA_WG_FACTORED && mode != VELORA_WG_EXPLICIT))
+        return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(dY, dy_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(dW, dw_dtype) ||
+        !elem_aligned(v, VELORA_F32))
+        return VELORA_ERR_ALIGNMENT;
+    if (!ws) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return VELORA_OK;
+}
+
+}  // namespace
+}  // namespace velora
+
+using namespace velora;
+
+extern "C" {
+
+int velora_version(void) { return 100; }
+
+const char* velora_status_string(int status)
+{
+    switch (status) {
+        case VELORA_OK: return "ok";
+        case VELORA_ERR_INVALID_ARG: return "invalid argument";
+        case VELORA_ERR_UNSUPPORTED: return "unsupported dtype or size";
+        case VELORA_ERR_ALIGNMENT: return "misaligned pointer";
+        case VELORA_ERR_WORKSPACE: return "workspace missing or too small";
+        case VELORA_ERR_DEGENERATE_V: return "sub-token sum has zero or non-finite length";
+        case VELORA_ERR_TIMEOUT: return "device-side wait timed out";
+        case VELORA_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
+{
+    if (N < 0 || D < 1 || Dsub < 1 || Dsub > D || Dsub > VELORA_MAX_DSUB) return 0;
+    switch (op) {
+        case VELORA_OP_INIT_V: return init_v_workspace_bytes(Dsub);
+        case VELORA_OP_WEIGHT_GRAD_FACTORED:
+        case VELORA_OP_LINEAR_BACKWARD_FACTORED: return O < 1 ? 0 : factored_bytes(N, D, O, Dsub);
+        case VELORA_OP_WEIGHT_GRAD_EXPLICIT:
+        case VELORA_OP_LINEAR_BACKWARD_EXPLICIT: return xhat_bytes(N, D);
+        case VELORA_OP_LINEAR_FORWARD: return 0;
+        default: return 0;
+    }
+}
+
+int velora_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                  float* v, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!X || !v) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (ldx < D) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(X, x_dtype) || !elem_aligned(v, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    if (N == 0) return VELORA_ERR_DEGENERATE_V;
+    return launch_init_v(X, x_dtype, N, D, ldx, Dsub, v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                    const float* v, void* Z, int z_dtype, int64_t ldz, void* stream)
+{
+    if (!X || !v || !Z) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (ldx < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(X, x_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
+        return VELORA_ERR_ALIGNMENT;
+    if (N == 0) return VELORA_OK;
+    return launch_compress(X, x_dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, static_cast<cudaStream_t>(stream));
+}
+
+int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
+                       const float* v, void* Xhat, int x_dtype, int64_t ldxhat, void* stream)
+{
+    if (!Z || !v || !Xhat) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (ldxhat < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(Xhat, x_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
+        return VELORA_ERR_ALIGNMENT;
+    if (N == 0) return VELORA_OK;
+    return launch_reconstruct(Z, z_dtype, ldz, N, D, Dsub, v, Xhat, x_dtype, ldxhat,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int velora_weight_grad(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                       const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                       void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
+                       void* ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_weight_grad_args(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
+                                    dW, dw_dtype, lddw, beta, mode, ws);
+    if (rc != VELORA_OK) return rc;
+    const size_t need = velora_workspace_bytes(mode == VELORA_WG_FACTORED ? VELORA_OP_WEIGHT_GRAD_FACTORED
+                                                                          : VELORA_OP_WEIGHT_GRAD_EXPLICIT,
+                                               N, D, O, Dsub);
+    if (ws_bytes < need) return VELORA_ERR_WORKSPACE;
+    return weight_grad_impl(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub, dW, dw_dtype, lddw,
+                            beta, mode, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
+                          void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
+                          int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
+                          void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    if (!X || !W || !v || !Y || !Z) return VELORA_ERR_INVALID_ARG;
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (ldx < D || ldw < D || ldy < O || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(X, dtype) || !elem_aligned(W, dtype) || !elem_aligned(Y, dtype) ||
+        !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
+        return VELORA_ERR_ALIGNMENT;
+    if (N == 0) return VELORA_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = launch_linear_forward_tc(X, ldx, W, ldw, v, Y, ldy, Z, z_dtype, ldz, dtype, N, D, O, Dsub, s);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    rc = launch_gemm_simt(X, dtype, ldx, 1, W, dtype, ldw, 1, Y, dtype, ldy, 0, N, O, D, s);
+    if (rc != VELORA_OK) return rc;
+    return launch_compress(X, dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, s);
+}
+
+int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t ldw,
+                           const void* Z, int z_dtype, int64_t ldz, const float* v,
+                           void* dX, int64_t lddx, void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
+                           int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
+                           void* ws, size_t ws_bytes, void* stream)
+{
+    if (!dY) return VELORA_ERR_INVALID_ARG;
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (lddy < O) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(dY, dtype)) return VELORA_ERR_ALIGNMENT;
+    if (dX) {
+        if (!W) return VELORA_ERR_INVALID_ARG;
+        if (ldw < D || lddx < D) return VELORA_ERR_INVALID_ARG;
+        if (!elem_aligned(W, dtype) || !elem_aligned(dX, dtype)) return VELORA_ERR_ALIGNMENT;
+    }
+    if (dW) {
+        rc = check_weight_grad_args(dY, dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
+                                    dW, dw_dtype, lddw, beta, mode, ws);
+        if (rc != VELORA_OK) return rc;
+        const size_t need = velora_workspace_bytes(mode == VELORA_WG_FACTORED ? VELORA_OP_LINEAR_BACKWARD_FACTORED
+                                                                              : VELORA_OP_LINEAR_BACKWARD_EXPLICIT,
+                                                   N, D, O, Dsub);
+        if (ws_bytes < need) return VELORA_ERR_WORKSPACE;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (dX && N > 0) {
+        rc = launch_gemm_tc(GEMM_NN_K_MN, dY, lddy, W, ldw, dX, dtype, lddx, 0, N, D, O, dtype, s);
+        if (rc == VELORA_ERR_UNSUPPORTED)
+            rc = launch_gemm_simt(dY, dtype, lddy, 1, W, dtype, 1, ldw, dX, dtype, lddx, 0, N, D, O, s);
+        if (rc != VELORA_OK) return rc;
+    }
+    if (dW)
+        return weight_grad_impl(dY, dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub, dW, dw_dtype, lddw,
+                                beta, mode, ws, ws_bytes, s);
+    return VELORA_OK;
+}
+
+}  // extern "C"

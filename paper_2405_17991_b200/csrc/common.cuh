@@ -1,0 +1,68 @@
+// Shared declarations of the VeLoRA CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "velora.h"
+
+namespace velora {
+
+constexpr int kStreamThreads = 256;       // CTA size of the streaming kernels
+constexpr int kStreamCtasPerSm = 8;       // resident CTAs per SM they are sized for
+constexpr int kInitVMaxCtas = 1184;       // rows of the init_v partial-sum scratch (148 SMs x 8)
+constexpr size_t kStatusBytes = 256;      // status word + padding at the head of a workspace
+
+struct DeviceInfo {
+    int sm_count;
+    int smem_optin;
+};
+// Attributes of the current device (cached per device ordinal).
+int device_info(DeviceInfo* out);
+
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : 4; }
+inline bool valid_dtype(int dt) { return dt == VELORA_F32 || dt == VELORA_BF16; }
+
+// ---- streaming kernels (stream_kernels.cu) ----
+int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
+size_t init_v_workspace_bytes(int Dsub);
+int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                    const float* v, void* Z, int z_dtype, int64_t ldz, cudaStream_t stream);
+int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
+                       const float* v, void* Xhat, int x_dtype, int64_t ldxhat, cudaStream_t stream);
+
+// ---- GEMMs ----
+// C[m, n] = sum_k A(m, k) * B(n, k) with element strides; fp32 accumulation on CUDA cores.
+// Serves the all-fp32 case and shapes the tensor-core path does not take.
+int launch_gemm_simt(const void* A, int a_dtype, int64_t a_sm, int64_t a_sk,
+                     const void* B, int b_dtype, int64_t b_sn, int64_t b_sk,
+                     void* C, int c_dtype, int64_t ldc, int beta,
+                     int64_t Mdim, int64_t Ndim, int64_t Kdim, cudaStream_t stream);
+
+// dW[o, m*Dsub + j] = beta*dW + P[o, m] * v[j] with P[O, M] fp32 (expansion after a CUDA-core P = dY^T Z).
+int launch_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
+                    void* dW, int dw_dtype, int64_t lddw, int beta, cudaStream_t stream);
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static __device__ __forceinline__ float load(const float* p) { return *p; }
+    static __device__ __forceinline__ void store(float* p, float x) { *p = x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static __device__ __forceinline__ float load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+};
+
+}  // namespace velora

@@ -1,0 +1,594 @@
+// HBM-bound streaming kernels of the VeLoRA path: init_v, compress, reconstruct
+// (arxiv 2405.17991, Section 3.1 Eq. 1 / Eq. 2, Section 3.2 initialisation).
+//
+// Vector kernels.  A row of X is a sequence of 16-byte chunks (8 bf16).  A
+// sub-token of length Dsub = 8*L is covered by LPS = min(L, 32) adjacent lanes,
+// each lane owning CH = L / LPS chunks, so a warp instruction reads one
+// contiguous 512-byte span.  Work items (row, m, lane-in-group) are numbered
+// row-major and walked with a grid-wide stride that is a multiple of 32: a
+// thread therefore keeps the same position inside its sub-token for the whole
+// kernel and holds its slice of v in registers.  The walk carries (row, pos)
+// incrementally -- no division in the loop.  When Dsub does not divide D the
+// last sub-token's missing chunks are simply not loaded (zero extension).
+//
+// Element kernels cover everything else (fp32 data, Dsub not a multiple of 8,
+// unaligned rows) with the same arithmetic, one element per lane.
+#include "common.cuh"
+
+namespace velora {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// Walks items tid, tid + S, tid + 2S, ... as (row, pos), pos in [0, items_per_row).
+struct ItemWalk {
+    int64_t row;
+    int pos;
+    int row_step, pos_step, ipr;
+    __device__ __forceinline__ void init(int items_per_row)
+    {
+        const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+        const int S = gridDim.x * blockDim.x;
+        ipr = items_per_row;
+        row = tid / ipr;
+        pos = tid - static_cast<int>(row) * ipr;
+        row_step = S / ipr;
+        pos_step = S - row_step * ipr;
+    }
+    __device__ __forceinline__ void advance()
+    {
+        pos += pos_step;
+        row += row_step;
+        if (pos >= ipr) { pos -= ipr; ++row; }
+    }
+};
+
+__device__ __forceinline__ void unpack8(const uint4& c, float (&x)[8])
+{
+    x[0] = bf16_lo(c.x); x[1] = bf16_hi(c.x);
+    x[2] = bf16_lo(c.y); x[3] = bf16_hi(c.y);
+    x[4] = bf16_lo(c.z); x[5] = bf16_hi(c.z);
+    x[6] = bf16_lo(c.w); x[7] = bf16_hi(c.w);
+}
+
+// Loads chunk `chunk` of a row, zeroing whatever lies at or beyond column D.
+__device__ __forceinline__ uint4 load_chunk(const uint4* row_ptr, int chunk, int D)
+{
+    const int col = chunk * 8;
+    uint4 c = make_uint4(0u, 0u, 0u, 0u);
+    if (col < D) {
+        c = __ldg(row_ptr + chunk);
+        if (col + 8 > D) {                       // ragged end of a row whose width is not a multiple of 8
+            const int keep = D - col;            // 1..7 valid elements
+            uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (2 * i >= keep) w[i] = 0u;
+                else if (2 * i + 1 >= keep) w[i] &= 0x0000ffffu;
+            }
+            c = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+    return c;
+}
+
+template <typename ZT> __device__ __forceinline__ void store_z(ZT* p, float z);
+template <> __device__ __forceinline__ void store_z<float>(float* p, float z) { *p = z; }
+template <> __device__ __forceinline__ void store_z<__nv_bfloat16>(__nv_bfloat16* p, float z) { *p = __float2bfloat16_rn(z); }
+
+// ------------------------------------------------------------------ compress (vector)
+template <int LPS, int CH, int U, typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+compress_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldx_chunks, int M,
+                    const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz)
+{
+    constexpr int L = LPS * CH;                  // chunks per sub-token
+    const int q = threadIdx.x & (LPS - 1);       // fixed position inside the sub-token
+    float vr[CH][8];
+#pragma unroll
+    for (int i = 0; i < CH; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
+
+    ItemWalk w;
+    w.init(M * LPS);
+    while (__any_sync(kFull, w.row < N)) {
+        uint4 data[U][CH];
+        int64_t rows[U];
+        int ms[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            rows[u] = w.row;
+            ms[u] = w.pos / LPS;                 // LPS is a power of two
+            const bool valid = w.row < N;
+            const uint4* rp = X + w.row * ldx_chunks;
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+                data[u][i] = valid ? load_chunk(rp, ms[u] * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
+            w.advance();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                float x[8];
+                unpack8(data[u][i], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc = fmaf(x[e], vr[i][e], acc);
+            }
+#pragma unroll
+            for (int off = LPS / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(kFull, acc, off);
+            if (q == 0 && rows[u] < N) store_z<ZT>(Z + rows[u] * ldz + ms[u], acc);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ reconstruct (vector, bf16 out)
+template <typename ZT> __device__ __forceinline__ float load_z(const ZT* p);
+template <> __device__ __forceinline__ float load_z<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float load_z<__nv_bfloat16>(const __nv_bfloat16* p)
+{
+    return __bfloat162float(*p);
+}
+
+__device__ __forceinline__ void store_chunk_bf16(uint4* row_ptr, __nv_bfloat16* row_elems, int chunk, int D,
+                                                 const float (&y)[8])
+{
+    const int col = chunk * 8;
+    if (col + 8 <= D) {
+        uint4 o;
+        o.x = pack_bf16x2(y[0], y[1]);
+        o.y = pack_bf16x2(y[2], y[3]);
+        o.z = pack_bf16x2(y[4], y[5]);
+        o.w = pack_bf16x2(y[6], y[7]);
+        __stcs(row_ptr + chunk, o);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (col + e < D) row_elems[col + e] = __float2bfloat16_rn(y[e]);
+    }
+}
+
+template <int LPS, int CH, int U, typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+reconstruct_vec_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D, int M,
+                       const float* __restrict__ v, uint4* __restrict__ Xhat, int64_t ldx_chunks)
+{
+    constexpr int L = LPS * CH;
+    const int q = threadIdx.x & (LPS - 1);
+    float vr[CH][8];
+#pragma unroll
+    for (int i = 0; i < CH; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
+
+    ItemWalk w;
+    w.init(M * LPS);
+    while (w.row < N) {
+        float z[U];
+        int64_t rows[U];
+        int ms[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            rows[u] = w.row;
+            ms[u] = w.pos / LPS;
+            z[u] = (w.row < N) ? load_z<ZT>(Z + w.row * ldz + ms[u]) : 0.f;
+            w.advance();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (rows[u] < N) {
+                uint4* rp = Xhat + rows[u] * ldx_chunks;
+                __nv_bfloat16* re = reinterpret_cast<__nv_bfloat16*>(rp);
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    float y[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) y[e] = z[u] * vr[i][e];
+                    const int chunk = ms[u] * L + q + LPS * i;
+                    if (chunk * 8 < D) store_chunk_bf16(rp, re, chunk, D, y);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ init_v (vector): per-CTA partial sums
+template <int LPS, int CH, int U>
+__global__ void __launch_bounds__(kStreamThreads)
+init_v_partial_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldx_chunks, int M,
+                          float* __restrict__ partials /* [gridDim.x][8*L] */)
+{
+    constexpr int L = LPS * CH;
+    constexpr int W = 8 * CH;                    // accumulators per thread
+    const int q = threadIdx.x & (LPS - 1);
+    float acc[CH][8];
+#pragma unroll
+    for (int i = 0; i < CH; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[i][e] = 0.f;
+
+    ItemWalk w;
+    w.init(M * LPS);
+    while (w.row < N) {
+        uint4 data[U][CH];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool valid = w.row < N;
+            const uint4* rp = X + w.row * ldx_chunks;
+            const int m = w.pos / LPS;
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+                data[u][i] = valid ? load_chunk(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
+            w.advance();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                float x[8];
+                unpack8(data[u][i], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[i][e] += x[e];
+            }
+    }
+
+    // Fixed-order reduction over the threads of the CTA that share a position q.
+    extern __shared__ float sacc[];              // [kStreamThreads][W]
+#pragma unroll
+    for (int i = 0; i < CH; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sacc[threadIdx.x * W + i * 8 + e] = acc[i][e];
+    __syncthreads();
+    for (int j = threadIdx.x; j < 8 * L; j += kStreamThreads) {
+        const int chunk = j >> 3, e = j & 7;
+        const int qq = chunk % LPS, i = chunk / LPS;
+        float s = 0.f;
+        for (int t = qq; t < kStreamThreads; t += LPS) s += sacc[t * W + i * 8 + e];
+        partials[static_cast<int64_t>(blockIdx.x) * (8 * L) + j] = s;
+    }
+}
+
+// ------------------------------------------------------------------ init_v (element-wise) partial sums
+// CTA b owns rows [b*rows_per_cta, ...).  For each block of up to 256 positions j, thread t adds
+// X[row, m*Dsub + j] over its rows and over m = slot, slot + slots, ...; slots share a position and are
+// summed in fixed order through shared memory.
+template <typename XT>
+__global__ void __launch_bounds__(kStreamThreads)
+init_v_partial_elem_kernel(const XT* __restrict__ X, int64_t N, int D, int64_t ldx, int Dsub, int M,
+                           int64_t rows_per_cta, float* __restrict__ partials /* [gridDim.x][Dsub] */)
+{
+    __shared__ float sred[kStreamThreads];
+    const int64_t r0 = blockIdx.x * rows_per_cta;
+    const int64_t r1 = (r0 + rows_per_cta < N) ? r0 + rows_per_cta : N;
+    for (int j0 = 0; j0 < Dsub; j0 += kStreamThreads) {
+        const int width = (Dsub - j0 < kStreamThreads) ? Dsub - j0 : kStreamThreads;
+        const int slots = kStreamThreads / width;
+        const int j = j0 + threadIdx.x % width;
+        const int slot = threadIdx.x / width;
+        float acc = 0.f;
+        if (slot < slots)
+            for (int64_t r = r0; r < r1; ++r)
+                for (int m = slot; m < M; m += slots) {
+                    const int d = m * Dsub + j;
+                    if (d < D) acc += Elem<XT>::load(X + r * ldx + d);
+                }
+        sred[threadIdx.x] = acc;
+        __syncthreads();
+        if (threadIdx.x < width) {
+            float s = 0.f;
+            for (int k = 0; k < slots; ++k) s += sred[k * width + threadIdx.x];
+            partials[static_cast<int64_t>(blockIdx.x) * Dsub + j] = s;
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ init_v finalize: one CTA
+// s[j] = sum over CTAs (fixed order, fp64), norm, v = s / ||s||.  status[0] = 0 ok, 1 degenerate.
+__global__ void __launch_bounds__(kStreamThreads)
+init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int Dsub,
+                       float* __restrict__ v, int* __restrict__ status)
+{
+    __shared__ double s_sum[VELORA_MAX_DSUB];
+    __shared__ double s_red[kStreamThreads];
+    __shared__ double s_norm;
+    double sq = 0.0;
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) {
+        double s = 0.0;
+        for (int b = 0; b < num_partials; ++b) s += static_cast<double>(partials[static_cast<int64_t>(b) * Dsub + j]);
+        s_sum[j] = s;
+        sq += s * s;
+    }
+    s_red[threadIdx.x] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < kStreamThreads; ++i) t += s_red[i];
+        s_norm = sqrt(t);
+    }
+    __syncthreads();
+    const double norm = s_norm;
+    const bool ok = (norm > 0.0) && isfinite(norm);
+    if (threadIdx.x == 0) status[0] = ok ? 0 : 1;
+    if (ok)
+        for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) v[j] = static_cast<float>(s_sum[j] / norm);
+}
+
+// ------------------------------------------------------------------ compress / reconstruct (element-wise)
+template <typename XT, typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+compress_elem_kernel(const XT* __restrict__ X, int64_t N, int D, int64_t ldx, int Dsub, int M,
+                     const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = static_cast<int64_t>(gridDim.x) * (kStreamThreads / 32);
+    const int64_t total = N * M;
+    for (int64_t g = static_cast<int64_t>(blockIdx.x) * (kStreamThreads / 32) + (threadIdx.x >> 5); g < total; g += warps) {
+        const int64_t row = g / M;
+        const int m = static_cast<int>(g - row * M);
+        const XT* xp = X + row * ldx + static_cast<int64_t>(m) * Dsub;
+        const int len = (D - m * Dsub < Dsub) ? D - m * Dsub : Dsub;
+        float acc = 0.f;
+        for (int j = lane; j < len; j += 32) acc = fmaf(Elem<XT>::load(xp + j), __ldg(v + j), acc);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(kFull, acc, off);
+        if (lane == 0) store_z<ZT>(Z + row * ldz + m, acc);
+    }
+}
+
+template <typename ZT, typename XT>
+__global__ void __launch_bounds__(kStreamThreads)
+reconstruct_elem_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D, int Dsub,
+                        const float* __restrict__ v, XT* __restrict__ Xhat, int64_t ldx)
+{
+    const int64_t total = N * D;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; idx < total; idx += stride) {
+        const int64_t row = idx / D;
+        const int d = static_cast<int>(idx - row * D);
+        const int m = d / Dsub;
+        const int j = d - m * Dsub;
+        Elem<XT>::store(Xhat + row * ldx + d, load_z<ZT>(Z + row * ldz + m) * __ldg(v + j));
+    }
+}
+
+// P[O, M] fp32 expanded to dW[o, m*Dsub + j] = beta*dW + P[o, m] v[j].
+template <typename WT>
+__global__ void __launch_bounds__(kStreamThreads)
+expand_p_kernel(const float* __restrict__ P, int64_t ldp, const float* __restrict__ v, int64_t O, int D, int Dsub,
+                WT* __restrict__ dW, int64_t lddw, int beta)
+{
+    const int64_t total = O * D;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; idx < total; idx += stride) {
+        const int64_t o = idx / D;
+        const int d = static_cast<int>(idx - o * D);
+        const int m = d / Dsub;
+        const int j = d - m * Dsub;
+        float r = __ldg(P + o * ldp + m) * __ldg(v + j);
+        if (beta) r += Elem<WT>::load(dW + o * lddw + d);
+        Elem<WT>::store(dW + o * lddw + d, r);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+struct VecShape {
+    bool ok;
+    int lps, ch, u;
+};
+
+// Vector kernels need Dsub = 8 * L with L a power of two up to 128.
+VecShape vec_shape(int Dsub)
+{
+    VecShape s{false, 0, 0, 0};
+    if (Dsub % 8) return s;
+    const int L = Dsub / 8;
+    if (L < 1 || L > 128 || (L & (L - 1))) return s;
+    s.ok = true;
+    s.lps = L < 32 ? L : 32;
+    s.ch = L / s.lps;
+    s.u = s.ch == 1 ? 4 : (s.ch == 2 ? 2 : 1);
+    return s;
+}
+
+bool rows_vectorisable(const void* p, int64_t ld_elems)
+{
+    return aligned16(p) && (ld_elems % 8 == 0);
+}
+
+int stream_grid(int64_t items, int per_thread, int* grid)
+{
+    DeviceInfo di;
+    const int rc = device_info(&di);
+    if (rc != VELORA_OK) return rc;
+    int64_t ctas = ceil_div64(items, static_cast<int64_t>(kStreamThreads) * per_thread);
+    const int64_t cap = static_cast<int64_t>(di.sm_count) * kStreamCtasPerSm;
+    if (ctas > cap) ctas = cap;
+    if (ctas < 1) ctas = 1;
+    *grid = static_cast<int>(ctas);
+    return VELORA_OK;
+}
+
+int check_launch()
+{
+    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+}
+
+// Largest number of rows one vector launch may take so that item counts stay below 2^30.
+int64_t max_rows_per_launch(int items_per_row)
+{
+    return (static_cast<int64_t>(1) << 30) / items_per_row;
+}
+
+#define VELORA_DISPATCH_VEC(SHAPE, KERNEL_CALL)                                              \
+    switch ((SHAPE).lps * 8 + (SHAPE).ch) {                                                  \
+        case 1 * 8 + 1: { KERNEL_CALL(1, 1, 4); break; }                                     \
+        case 2 * 8 + 1: { KERNEL_CALL(2, 1, 4); break; }                                     \
+        case 4 * 8 + 1: { KERNEL_CALL(4, 1, 4); break; }                                     \
+        case 8 * 8 + 1: { KERNEL_CALL(8, 1, 4); break; }                                     \
+        case 16 * 8 + 1: { KERNEL_CALL(16, 1, 4); break; }                                   \
+        case 32 * 8 + 1: { KERNEL_CALL(32, 1, 4); break; }                                   \
+        case 32 * 8 + 2: { KERNEL_CALL(32, 2, 2); break; }                                   \
+        case 32 * 8 + 4: { KERNEL_CALL(32, 4, 1); break; }                                   \
+        default: return VELORA_ERR_UNSUPPORTED;                                              \
+    }
+
+}  // namespace
+
+size_t init_v_workspace_bytes(int Dsub)
+{
+    return kStatusBytes + static_cast<size_t>(kInitVMaxCtas) * static_cast<size_t>(Dsub) * sizeof(float);
+}
+
+int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
+    int* status = static_cast<int*>(ws);
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
+    const int M = static_cast<int>(ceil_div64(D, Dsub));
+    const VecShape vs = vec_shape(Dsub);
+    int num_partials = 0;
+
+    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx) &&
+        N <= max_rows_per_launch(M * vs.lps)) {
+        const int64_t items = N * M * vs.lps;
+        int grid = 0;
+        int rc = stream_grid(items, vs.u, &grid);
+        if (rc != VELORA_OK) return rc;
+        if (grid > kInitVMaxCtas) grid = kInitVMaxCtas;
+        num_partials = grid;
+        const size_t smem = static_cast<size_t>(kStreamThreads) * 8 * vs.ch * sizeof(float);
+#define CALL_INIT(LPS, CH, U)                                                                             \
+        init_v_partial_vec_kernel<LPS, CH, U><<<grid, kStreamThreads, smem, stream>>>(                    \
+            static_cast<const uint4*>(X), N, static_cast<int>(D), ldx / 8, M, partials)
+        VELORA_DISPATCH_VEC(vs, CALL_INIT)
+#undef CALL_INIT
+    } else {
+        DeviceInfo di;
+        int rc = device_info(&di);
+        if (rc != VELORA_OK) return rc;
+        int64_t grid = static_cast<int64_t>(di.sm_count) * 4;
+        if (grid > kInitVMaxCtas) grid = kInitVMaxCtas;
+        if (grid > N) grid = N;
+        const int64_t rows_per_cta = ceil_div64(N, grid);
+        grid = ceil_div64(N, rows_per_cta);
+        num_partials = static_cast<int>(grid);
+        if (x_dtype == VELORA_BF16)
+            init_v_partial_elem_kernel<__nv_bfloat16><<<static_cast<int>(grid), kStreamThreads, 0, stream>>>(
+                static_cast<const __nv_bfloat16*>(X), N, static_cast<int>(D), ldx, Dsub, M, rows_per_cta, partials);
+        else
+            init_v_partial_elem_kernel<float><<<static_cast<int>(grid), kStreamThreads, 0, stream>>>(
+                static_cast<const float*>(X), N, static_cast<int>(D), ldx, Dsub, M, rows_per_cta, partials);
+    }
+    if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(partials, num_partials, Dsub, v, status);
+    if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+
+    int host_status = -1;
+    if (cudaMemcpyAsync(&host_status, status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return VELORA_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (host_status == 0) return VELORA_OK;
+    return host_status == 1 ? VELORA_ERR_DEGENERATE_V : VELORA_ERR_CUDA;
+}
+
+int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                    const float* v, void* Z, int z_dtype, int64_t ldz, cudaStream_t stream)
+{
+    const int M = static_cast<int>(ceil_div64(D, Dsub));
+    const VecShape vs = vec_shape(Dsub);
+    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx)) {
+        const int64_t step = max_rows_per_launch(M * vs.lps);
+        for (int64_t r0 = 0; r0 < N; r0 += step) {
+            const int64_t n = (N - r0 < step) ? N - r0 : step;
+            int grid = 0;
+            int rc = stream_grid(n * M * vs.lps, vs.u, &grid);
+            if (rc != VELORA_OK) return rc;
+            const uint4* xp = static_cast<const uint4*>(X) + r0 * (ldx / 8);
+#define CALL_COMPRESS(LPS, CH, U)                                                                         \
+            if (z_dtype == VELORA_F32)                                                                    \
+                compress_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(              \
+                    xp, n, static_cast<int>(D), ldx / 8, M, v, static_cast<float*>(Z) + r0 * ldz, ldz);   \
+            else                                                                                          \
+                compress_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(      \
+                    xp, n, static_cast<int>(D), ldx / 8, M, v, static_cast<__nv_bfloat16*>(Z) + r0 * ldz, ldz)
+            VELORA_DISPATCH_VEC(vs, CALL_COMPRESS)
+#undef CALL_COMPRESS
+            if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+        }
+        return VELORA_OK;
+    }
+    int grid = 0;
+    int rc = stream_grid(N * M * 32, 1, &grid);
+    if (rc != VELORA_OK) return rc;
+#define CALL_ELEM(XT, ZT)                                                                                 \
+    compress_elem_kernel<XT, ZT><<<grid, kStreamThreads, 0, stream>>>(                                    \
+        static_cast<const XT*>(X), N, static_cast<int>(D), ldx, Dsub, M, v, static_cast<ZT*>(Z), ldz)
+    if (x_dtype == VELORA_BF16 && z_dtype == VELORA_F32) CALL_ELEM(__nv_bfloat16, float);
+    else if (x_dtype == VELORA_BF16) CALL_ELEM(__nv_bfloat16, __nv_bfloat16);
+    else if (z_dtype == VELORA_F32) CALL_ELEM(float, float);
+    else CALL_ELEM(float, __nv_bfloat16);
+#undef CALL_ELEM
+    return check_launch();
+}
+
+int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
+                       const float* v, void* Xhat, int x_dtype, int64_t ldxhat, cudaStream_t stream)
+{
+    const int M = static_cast<int>(ceil_div64(D, Dsub));
+    const VecShape vs = vec_shape(Dsub);
+    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(Xhat, ldxhat)) {
+        const int64_t step = max_rows_per_launch(M * vs.lps);
+        for (int64_t r0 = 0; r0 < N; r0 += step) {
+            const int64_t n = (N - r0 < step) ? N - r0 : step;
+            int grid = 0;
+            int rc = stream_grid(n * M * vs.lps, vs.u, &grid);
+            if (rc != VELORA_OK) return rc;
+            uint4* xp = static_cast<uint4*>(Xhat) + r0 * (ldxhat / 8);
+#define CALL_RECON(LPS, CH, U)                                                                            \
+            if (z_dtype == VELORA_F32)                                                                    \
+                reconstruct_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(           \
+                    static_cast<const float*>(Z) + r0 * ldz, ldz, n, static_cast<int>(D), M, v, xp, ldxhat / 8); \
+            else                                                                                          \
+                reconstruct_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(   \
+                    static_cast<const __nv_bfloat16*>(Z) + r0 * ldz, ldz, n, static_cast<int>(D), M, v, xp, ldxhat / 8)
+            VELORA_DISPATCH_VEC(vs, CALL_RECON)
+#undef CALL_RECON
+            if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+        }
+        return VELORA_OK;
+    }
+    int grid = 0;
+    int rc = stream_grid(N * D, 4, &grid);
+    if (rc != VELORA_OK) return rc;
+#define CALL_ELEM(ZT, XT)                                                                                 \
+    reconstruct_elem_kernel<ZT, XT><<<grid, kStreamThreads, 0, stream>>>(                                 \
+        static_cast<const ZT*>(Z), ldz, N, static_cast<int>(D), Dsub, v, static_cast<XT*>(Xhat), ldxhat)
+    if (z_dtype == VELORA_F32 && x_dtype == VELORA_BF16) CALL_ELEM(float, __nv_bfloat16);
+    else if (z_dtype == VELORA_F32) CALL_ELEM(float, float);
+    else if (x_dtype == VELORA_BF16) CALL_ELEM(__nv_bfloat16, __nv_bfloat16);
+    else CALL_ELEM(__nv_bfloat16, float);
+#undef CALL_ELEM
+    return check_launch();
+}
+
+int launch_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
+                    void* dW, int dw_dtype, int64_t lddw, int beta, cudaStream_t stream)
+{
+    int grid = 0;
+    int rc = stream_grid(O * D, 4, &grid);
+    if (rc != VELORA_OK) return rc;
+    if (dw_dtype == VELORA_BF16)
+        expand_p_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(
+            P, ldp, v, O, static_cast<int>(D), Dsub, static_cast<__nv_bfloat16*>(dW), lddw, beta);
+    else
+        expand_p_kernel<float><<<grid, kStreamThreads, 0, stream>>>(
+            P, ldp, v, O, static_cast<int>(D), Dsub, static_cast<float*>(dW), lddw, beta);
+    return check_launch();
+}
+
+}  // namespace velora
