@@ -1,0 +1,266 @@
+"""GPU parity: every C-ABI entry point against the fp64 CPU oracle on the same seeded inputs.
+
+Tolerances (derived from the arithmetic: bf16 inputs, fp32 products and sums): Z and Xhat within
+1e-3 norm-wise relative error; dW, Y, dX within 1e-2 relative Frobenius error.  An output stored in
+bf16 or fp32 is compared with the oracle's float64 result rounded once to that type.  Each entry
+point is checked on its own inputs: reconstruct and weight_grad oracles take the very Z buffer the
+GPU call receives.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import velora_inputs as vi
+from _util import TOL_GEMM, TOL_Z, assert_matches, rel_err, to_f64
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def vl():
+    import paper_2405_17991_b200 as pkg
+    pkg.lib()                      # raises if the CUDA library is missing: no fallback
+    return pkg
+
+
+def _distinct_D(cfg):
+    seen, out = set(), []
+    for i, layer in enumerate(cfg.layers):
+        if layer.D not in seen:
+            seen.add(layer.D)
+            out.append(i)
+    return out
+
+
+STREAM_CASES = [(c, li, ds) for c in (2, 3, 4, 5) for li in _distinct_D(vi.CONFIGS[c]) for ds in vi.CONFIGS[c].Dsubs]
+
+
+# ------------------------------------------------------------------ config 1: everything, brute force
+def test_config1_fp32_every_entry_point(vl):
+    cfg = vi.CONFIGS[1]
+    Dsub = cfg.Dsubs[0]
+    Xa, Wa, dYa = vi.make_X(cfg, 0), vi.make_W(cfg, 0), vi.make_dY(cfg, 0)
+    X, W, dY = Xa.torch(DEV), Wa.torch(DEV), dYa.torch(DEV)
+    N, D = X.shape
+    v = vl.velora_init_v(X, Dsub)
+    v_ref = oracle.init_v(Xa.f64(), Dsub)
+    assert rel_err(to_f64(v), v_ref) < 1e-5
+    assert abs(float(torch.linalg.vector_norm(v.double())) - 1.0) < 1e-6
+    v64 = to_f64(v)                                   # later steps use the fp32 v the GPU holds
+    Z = vl.velora_compress(X, v)
+    assert_matches(Z, oracle.compress(Xa.f64(), v64), 1e-5, "Z", ulps=16)
+    Xhat = vl.velora_reconstruct(Z, v, D, x_dtype=torch.float32)
+    assert_matches(Xhat, oracle.reconstruct(to_f64(Z), v64, D), 1e-6, "Xhat", ulps=2)
+    dW_ref = oracle.weight_grad(dYa.f64(), to_f64(Z), v64, D)            # brute force
+    for mode in (vl.WG_FACTORED, vl.WG_EXPLICIT):
+        dW = vl.velora_weight_grad(dY, Z, v, D, mode=mode)
+        assert_matches(dW, dW_ref, 1e-5, "dW mode %d" % mode)
+    Y, Z2 = vl.velora_linear_forward(X, W, v)
+    assert_matches(Y, oracle.linear_forward(Xa.f64(), Wa.f64()), 1e-5, "Y")
+    assert torch.equal(Z2, Z)
+    dX, dW = vl.velora_linear_backward(dY, W, Z, v)
+    assert_matches(dX, oracle.input_grad(dYa.f64(), Wa.f64()), 1e-5, "dX")
+    assert_matches(dW, dW_ref, 1e-5, "dW (linear_backward)")
+
+
+# ------------------------------------------------------------------ streaming kernels, full size
+@pytest.mark.parametrize("c,li,Dsub", STREAM_CASES)
+def test_init_v_compress_reconstruct_full_size(vl, c, li, Dsub):
+    cfg = vi.CONFIGS[c]
+    Xa = vi.make_X(cfg, li)
+    X64 = Xa.f64()
+    N, D = Xa.shape
+    ld = -(-D // 8) * 8                               # rows padded to 16 bytes (D = 5461 -> 5464)
+    X = Xa.torch(DEV, ld=ld)
+    v = vl.velora_init_v(X, Dsub)
+    v_ref, s, norm = oracle.init_v(X64, Dsub, return_sum=True)
+    assert rel_err(to_f64(v), v_ref) < TOL_Z
+    v64 = to_f64(v)
+    Z = vl.velora_compress(X, v)
+    assert_matches(Z, oracle.compress(X64, v64), TOL_Z, "Z f32", ulps=None)
+    Zb = vl.velora_compress(X, v, z_dtype=torch.bfloat16)
+    assert_matches(Zb, oracle.compress(X64, v64), TOL_Z, "Z bf16", ulps=1)
+    for Zin in (Z, Zb):
+        Xhat = vl.velora_reconstruct(Zin, v, D)
+        assert_matches(Xhat, oracle.reconstruct(to_f64(Zin), v64, D), TOL_Z, "Xhat", ulps=1)
+    # properties that hold at any size: unit norm; sum of Z equals ||s||
+    assert abs(float(torch.linalg.vector_norm(v.double())) - 1.0) < 1e-5
+    assert abs(float(Z.double().sum()) - norm) < 1e-3 * norm + 1e-2 * np.sqrt(Z.numel())
+
+
+def test_unpadded_odd_rows_take_the_elementwise_kernels(vl):
+    cfg = vi.CONFIGS[4]
+    li = 6                                            # down projection: D = 5461, odd row pitch
+    Xa = vi.make_X(cfg, li, N=512)
+    X = Xa.torch(DEV)
+    assert X.stride(0) == 5461
+    v = vl.velora_init_v(X, 128)
+    assert rel_err(to_f64(v), oracle.init_v(Xa.f64(), 128)) < TOL_Z
+    v64 = to_f64(v)
+    Z = vl.velora_compress(X, v)
+    assert_matches(Z, oracle.compress(Xa.f64(), v64), TOL_Z, "Z")
+    Xhat = vl.velora_reconstruct(Z, v, 5461)
+    assert Xhat.stride(0) == 5461
+    assert_matches(Xhat, oracle.reconstruct(to_f64(Z), v64, 5461), TOL_Z, "Xhat", ulps=1)
+    # padded and unpadded layouts give the same numbers
+    Xp = Xa.torch(DEV, ld=5464)
+    Zp = vl.velora_compress(Xp, v)
+    assert rel_err(to_f64(Zp), to_f64(Z)) < 1e-5
+
+
+EDGE = [
+    # N, D, O, Dsub
+    (1, 64, 8, 64),        # one token, Dsub = D
+    (3, 8, 5, 1),          # Dsub = 1: exact
+    (129, 72, 24, 24),     # Dsub multiple of 8 but not a power of two
+    (77, 100, 17, 16),     # ragged tail: M = 7, last sub-token has 4 entries; D not a multiple of 8
+    (300, 1024, 40, 512),  # long sub-tokens (two chunks per lane)
+    (130, 2048, 16, 1024), # longest supported sub-token
+    (1000, 40, 33, 8),     # one chunk per sub-token
+    (257, 136, 130, 10),   # Dsub not a multiple of 8
+]
+
+
+@pytest.mark.parametrize("N,D,O,Dsub", EDGE)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_edge_shapes_all_entry_points(vl, N, D, O, Dsub, dtype):
+    case = vi.small_case(7000 + N + D, N, D, O, dtype=dtype, mean_offset=0.25)
+    Xa, Wa, dYa = case["X"], case["W"], case["dY"]
+    ld = -(-D // 8) * 8
+    X, W, dY = Xa.torch(DEV, ld=ld), Wa.torch(DEV, ld=ld), dYa.torch(DEV, ld=-(-O // 8) * 8)
+    v = vl.velora_init_v(X, Dsub)
+    assert rel_err(to_f64(v), oracle.init_v(Xa.f64(), Dsub)) < 1e-4
+    v64 = to_f64(v)
+    Z = vl.velora_compress(X, v)
+    Z_ref = oracle.compress(Xa.f64(), v64)
+    assert_matches(Z, Z_ref, TOL_Z, "Z")
+    out_dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    Xhat = vl.velora_reconstruct(Z, v, D, x_dtype=out_dt)
+    assert_matches(Xhat, oracle.reconstruct(to_f64(Z), v64, D), TOL_Z, "Xhat", ulps=1)
+    if Dsub == 1:
+        assert_matches(Xhat, Xa.f64(), 1e-6, "Xhat exact for Dsub=1")
+    dW_ref = oracle.weight_grad(dYa.f64(), to_f64(Z), v64, D)
+    for mode in (vl.WG_FACTORED, vl.WG_EXPLICIT):
+        for dw_dt in (out_dt, torch.float32):
+            dW = vl.velora_weight_grad(dY, Z, v, D, mode=mode, dw_dtype=dw_dt)
+            assert_matches(dW, dW_ref, TOL_GEMM, "dW")
+    Y, Z2 = vl.velora_linear_forward(X, W, v)
+    assert_matches(Y, oracle.linear_forward(Xa.f64(), Wa.f64()), TOL_GEMM, "Y")
+    assert_matches(Z2, Z_ref, TOL_Z, "Z from linear_forward")
+    dX, dW = vl.velora_linear_backward(dY, W, Z, v)
+    assert_matches(dX, oracle.input_grad(dYa.f64(), Wa.f64()), TOL_GEMM, "dX")
+    assert_matches(dW, dW_ref, TOL_GEMM, "dW")
+
+
+def test_gradient_accumulation_beta_one(vl):
+    case = vi.small_case(11, 200, 256, 96, dtype="bf16")
+    X, dY = case["X"].torch(DEV), case["dY"].torch(DEV)
+    v = vl.velora_init_v(X, 32)
+    Z = vl.velora_compress(X, v)
+    v64 = to_f64(v)
+    base = torch.randn(96, 256, device=DEV, generator=torch.Generator(DEV).manual_seed(5))
+    for mode in (vl.WG_FACTORED, vl.WG_EXPLICIT):
+        dW = base.clone()
+        vl.velora_weight_grad(dY, Z, v, 256, dW=dW, beta=1, mode=mode)
+        ref = oracle.weight_grad(case["dY"].f64(), to_f64(Z), v64, 256, dW0=to_f64(base))
+        assert_matches(dW, ref, TOL_GEMM, "dW accumulate")
+
+
+def test_empty_batch_and_degenerate_mean(vl):
+    X = torch.zeros((0, 64), dtype=torch.bfloat16, device=DEV)
+    v = torch.full((16,), 7.0, device=DEV)
+    Z = vl.velora_compress(X, v)
+    assert Z.shape == (0, 4)
+    with pytest.raises(vl.VeloraError) as e:
+        vl.velora_init_v(X, 16, v=v)
+    assert e.value.status == 5
+    Xz = torch.zeros((10, 64), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(vl.VeloraError) as e:
+        vl.velora_init_v(Xz, 16, v=v)
+    assert e.value.status == 5
+    assert torch.all(v == 7.0)                        # v untouched
+    Xc = torch.tensor([[1.0, -2.0, -1.0, 2.0]], dtype=torch.float32, device=DEV)
+    with pytest.raises(vl.VeloraError):
+        vl.velora_init_v(Xc, 2)
+    Xn = torch.full((4, 16), float("nan"), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(vl.VeloraError):
+        vl.velora_init_v(Xn, 8)
+
+
+def test_results_are_run_to_run_identical(vl):
+    cfg = vi.CONFIGS[2]
+    X, dY = vi.make_X(cfg, 6).torch(DEV), vi.make_dY(cfg, 6).torch(DEV)
+    W = vi.make_W(cfg, 6).torch(DEV)
+    outs = []
+    for _ in range(2):
+        v = vl.velora_init_v(X, 64)
+        Y, Z = vl.velora_linear_forward(X, W, v)
+        dX, dW = vl.velora_linear_backward(dY, W, Z, v)
+        outs.append((v, Y, Z, dX, dW))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    # a frozen v survives a save / reload: Z is bit-identical
+    v2 = outs[0][0].cpu().clone().to(DEV)
+    assert torch.equal(vl.velora_compress(X, v2), vl.velora_compress(X, outs[0][0]))
+
+
+# ------------------------------------------------------------------ weight gradient and dense products
+GEMM_CASES = [(c, li, ds) for c in (2, 3, 4, 5) for li in range(len(vi.CONFIGS[c].layers))
+              for ds in vi.CONFIGS[c].Dsubs
+              if vi.CONFIGS[c].layers[li].name in ("q", "up", "down", "qkv", "proj", "fc1", "fc2")]
+
+
+@pytest.mark.parametrize("c,li,Dsub", GEMM_CASES)
+def test_linear_forward_backward_configs(vl, c, li, Dsub):
+    """Full-size launches; the oracle checks Z in full and Y, dX, dW on seeded samples of rows
+    (dW in full where the factored oracle is cheap enough)."""
+    cfg = vi.CONFIGS[c]
+    layer = cfg.layers[li]
+    N, D, O = cfg.N, layer.D, layer.O
+    Xa, Wa, dYa = vi.make_X(cfg, li), vi.make_W(cfg, li), vi.make_dY(cfg, li)
+    ldD, ldO = -(-D // 8) * 8, -(-O // 8) * 8
+    X, W, dY = Xa.torch(DEV, ld=ldD), Wa.torch(DEV, ld=ldD), dYa.torch(DEV, ld=ldO)
+    v = vl.velora_init_v(X, Dsub)
+    v64 = to_f64(v)
+    Y, Z = vl.velora_linear_forward(X, W, v)
+    assert_matches(Z, oracle.compress(Xa.f64(), v64), TOL_Z, "Z (fused forward)")
+    rows = vi.sample_rows(cfg, li, N, 192)
+    W64 = Wa.f64()
+    assert_matches(Y[rows], oracle.linear_forward(Xa.rows(rows).f64(), W64), TOL_GEMM, "Y rows")
+    dX, dW = vl.velora_linear_backward(dY, W, Z, v)
+    assert_matches(dX[rows], oracle.input_grad(dYa.rows(rows).f64(), W64), TOL_GEMM, "dX rows")
+    Z64 = to_f64(Z)
+    dY64 = dYa.f64()
+    M = Z.shape[1]
+    if N * O * M <= 1.5e9:                              # the factored oracle over every output row
+        dW_ref = oracle.weight_grad(dY64, Z64, v64, D, factored=True)
+        dW_chk, sel = dW, slice(None)
+    else:                                               # seeded sample of output rows
+        sel = vi.sample_rows(cfg, li, O, 256, salt=2)
+        dW_ref = oracle.weight_grad(np.ascontiguousarray(dY64[:, sel]), Z64, v64, D, factored=True)
+        dW_chk = dW[sel]
+    assert_matches(dW_chk, dW_ref, TOL_GEMM, "dW factored")
+    orows = vi.sample_rows(cfg, li, O, 48 if N * D < 5e7 else 16, salt=1)
+    dW_bf = oracle.weight_grad(np.ascontiguousarray(dY64[:, orows]), Z64, v64, D)    # plain definition
+    assert_matches(dW[orows], dW_bf, TOL_GEMM, "dW rows vs brute force")
+    dW_ex = vl.velora_weight_grad(dY, Z, v, D, mode=vl.WG_EXPLICIT)
+    assert_matches(dW_ex[sel], dW_ref, TOL_GEMM, "dW explicit")
+    assert rel_err(to_f64(dW_ex), to_f64(dW)) < TOL_GEMM
+
+
+def test_chained_path_against_chained_oracle(vl):
+    """init_v -> compress -> weight_grad on the GPU against the same chain in fp64 (bf16 Z storage)."""
+    cfg = vi.CONFIGS[3]
+    li = 3
+    Xa, dYa = vi.make_X(cfg, li), vi.make_dY(cfg, li)
+    X, dY = Xa.torch(DEV), dYa.torch(DEV)
+    D = Xa.shape[1]
+    v = vl.velora_init_v(X, 32)
+    Z = vl.velora_compress(X, v, z_dtype=torch.bfloat16)
+    dW = vl.velora_weight_grad(dY, Z, v, D)
+    v_ref = oracle.init_v(Xa.f64(), 32)
+    dW_ref = oracle.weight_grad(dYa.f64(), oracle.compress(Xa.f64(), v_ref), v_ref, D, factored=True)
+    assert rel_err(to_f64(dW), dW_ref) < TOL_GEMM
