@@ -90,6 +90,18 @@ const char* velora_status_string(int status);
 size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub);
 
 /*
+ * Workspace header.  The first 256 bytes of every workspace are a status area; word 0 is a sticky
+ * device error flag that a kernel raises when one of its bounded waits (on a shared-memory barrier
+ * fed by a tile copy or by the tensor cores) gives up after one second instead of spinning for ever.
+ * velora_workspace_init zeroes the header (asynchronously, on `stream`): call it once after
+ * allocating a workspace.  velora_workspace_status synchronises `stream`, reads the flag and returns
+ * VELORA_OK or VELORA_ERR_TIMEOUT; outputs of a call that raised the flag are undefined.
+ * The paper has no counterpart: this is run-time hygiene of the implementation.
+ */
+int velora_workspace_init(void* ws, size_t ws_bytes, void* stream);
+int velora_workspace_status(const void* ws, void* stream);
+
+/*
  * Initialise the projection vector from a batch (Section 3.2, "Cheap
  * initialisation strategies": the average of the first batch's sub-tokens;
  * Section 3.1: v has unit length):
@@ -140,7 +152,7 @@ int velora_weight_grad(const void* dY, int dy_dtype, int64_t N, int64_t O, int64
  * `dtype` is the storage type of X, W and Y (bf16: tensor cores with fp32
  * accumulation; f32: CUDA cores).  Z as in velora_compress.  X itself need not
  * be kept by the caller afterwards: (Z, W, v) is all the backward needs.
- * ws: velora_workspace_bytes(VELORA_OP_LINEAR_FORWARD, ...) bytes (may be 0 / NULL).
+ * ws: velora_workspace_bytes(VELORA_OP_LINEAR_FORWARD, ...) bytes.
  */
 int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
                           void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
@@ -152,6 +164,7 @@ int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw
  *     dX[N, D] = dY W                  (exact; skipped when dX == NULL)
  *     dW[O, D] as velora_weight_grad   (skipped when dW == NULL)
  * `dtype` is the storage type of dY, W and dX.
+ * ws: velora_workspace_bytes(VELORA_OP_LINEAR_BACKWARD_{FACTORED,EXPLICIT}, ...) bytes, always required.
  */
 int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t ldw,
                            const void* Z, int z_dtype, int64_t ldz, const float* v,

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     OP_LINEAR_FORWARD, OP_WEIGHT_GRAD_EXPLICIT, OP_WEIGHT_GRAD_FACTORED, SIGNATURES, WG_EXPLICIT,
     WG_FACTORED, VeloraError, lib, num_subtokens, velora_compress, velora_init_v,
     velora_linear_backward, velora_linear_forward, velora_reconstruct, velora_status_string,
-    velora_version, velora_weight_grad, velora_workspace_bytes,
+    velora_version, velora_weight_grad, velora_workspace_alloc, velora_workspace_bytes,
+    velora_workspace_init, velora_workspace_status,
 )
 from .memory_model import saved_activation_bytes  # noqa: F401

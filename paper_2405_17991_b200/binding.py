@@ -29,6 +29,8 @@ SIGNATURES = {
     "velora_version": (_int, []),
     "velora_status_string": (ctypes.c_char_p, [_int]),
     "velora_workspace_bytes": (_sz, [_int, _i64, _i64, _i64, _int]),
+    "velora_workspace_init": (_int, [_p, _sz, _p]),
+    "velora_workspace_status": (_int, [_p, _p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_reconstruct": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
@@ -98,8 +100,25 @@ def _stream(stream) -> ctypes.c_void_p:
 
 def _ws(ws: Optional[torch.Tensor], need: int, device) -> torch.Tensor:
     if ws is None:
-        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        ws = velora_workspace_alloc(need, device)
     return ws
+
+
+def velora_workspace_alloc(nbytes: int, device) -> torch.Tensor:
+    """Device workspace of at least ``nbytes`` with its status header zeroed."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    velora_workspace_init(ws)
+    return ws
+
+
+def velora_workspace_init(ws: torch.Tensor, stream=None) -> None:
+    _check(lib().velora_workspace_init(ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream)),
+           "velora_workspace_init")
+
+
+def velora_workspace_status(ws: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream; 0 or ERR_TIMEOUT if a kernel's bounded wait expired."""
+    return int(lib().velora_workspace_status(ctypes.c_void_p(ws.data_ptr()), _stream(stream)))
 
 
 def _check(status: int, where: str):

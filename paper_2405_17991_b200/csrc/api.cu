@@ -46,7 +46,10 @@ int64_t round_up8(int64_t x) { return (x + 7) / 8 * 8; }
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
-size_t xhat_bytes(int64_t N, int64_t D) { return align256(static_cast<size_t>(N) * round_up8(D) * 4); }
+size_t xhat_bytes(int64_t N, int64_t D)
+{
+    return kStatusBytes + align256(static_cast<size_t>(N) * round_up8(D) * 4);
+}
 
 size_t factored_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
 {
@@ -62,11 +65,12 @@ int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t
                      void* ws, size_t ws_bytes, cudaStream_t stream)
 {
     const int64_t M = num_subtokens(D, Dsub);
+    int* status = static_cast<int*>(ws);                 // word 0: sticky device error flag
+    char* body = static_cast<char*>(ws) + kStatusBytes;
     if (mode == VELORA_WG_FACTORED) {
         if (ws_bytes < factored_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
-        char* body = static_cast<char*>(ws) + kStatusBytes;
         int rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
-                                       dW, dw_dtype, lddw, beta, body, ws_bytes - kStatusBytes, stream);
+                                       dW, dw_dtype, lddw, beta, body, ws_bytes - kStatusBytes, status, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
         // CUDA-core route: P[O, M] = dY^T Z, then the outer-product expansion.
         float* P = reinterpret_cast<float*>(body);
@@ -77,11 +81,11 @@ int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t
     // Explicit: Xhat into the workspace in dY's storage type, then dW = dY^T Xhat.
     if (ws_bytes < xhat_bytes(N, D)) return VELORA_ERR_WORKSPACE;
     const int64_t ldxh = round_up8(D);
-    int rc = launch_reconstruct(Z, z_dtype, ldz, N, D, Dsub, v, ws, dy_dtype, ldxh, stream);
+    int rc = launch_reconstruct(Z, z_dtype, ldz, N, D, Dsub, v, body, dy_dtype, ldxh, stream);
     if (rc != VELORA_OK) return rc;
-    rc = launch_gemm_tc(GEMM_TN_MN_MN, dY, lddy, ws, ldxh, dW, dw_dtype, lddw, beta, O, D, N, dy_dtype, stream);
+    rc = launch_gemm_tc(GEMM_TN_MN_MN, dY, lddy, body, ldxh, dW, dw_dtype, lddw, beta, O, D, N, dy_dtype, status, stream);
     if (rc != VELORA_ERR_UNSUPPORTED) return rc;
-    return launch_gemm_simt(dY, dy_dtype, 1, lddy, ws, dy_dtype, 1, ldxh, dW, dw_dtype, lddw, beta, O, D, N, stream);
+    return launch_gemm_simt(dY, dy_dtype, 1, lddy, body, dy_dtype, 1, ldxh, dW, dw_dtype, lddw, beta, O, D, N, stream);
 }
 
 int check_weight_grad_args(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
@@ -113,6 +117,24 @@ extern "C" {
 
 int velora_version(void) { return 100; }
 
+int velora_workspace_init(void* ws, size_t ws_bytes, void* stream)
+{
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return cudaMemsetAsync(ws, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? VELORA_OK
+                                                                                                   : VELORA_ERR_CUDA;
+}
+
+int velora_workspace_status(const void* ws, void* stream)
+{
+    if (!ws) return VELORA_ERR_WORKSPACE;
+    int word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return VELORA_ERR_CUDA;
+    return word == 0 ? VELORA_OK : VELORA_ERR_TIMEOUT;
+}
+
 const char* velora_status_string(int status)
 {
     switch (status) {
@@ -137,7 +159,7 @@ size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
         case VELORA_OP_LINEAR_BACKWARD_FACTORED: return O < 1 ? 0 : factored_bytes(N, D, O, Dsub);
         case VELORA_OP_WEIGHT_GRAD_EXPLICIT:
         case VELORA_OP_LINEAR_BACKWARD_EXPLICIT: return xhat_bytes(N, D);
-        case VELORA_OP_LINEAR_FORWARD: return 0;
+        case VELORA_OP_LINEAR_FORWARD: return kStatusBytes;
         default: return 0;
     }
 }
@@ -145,43 +167,43 @@ size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
 int velora_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
                   float* v, void* ws, size_t ws_bytes, void* stream)
 {
-    if (!X || !v) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
     if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (N == 0) return VELORA_ERR_DEGENERATE_V;      /* an empty batch has no mean; X may be NULL */
+    if (!X || !v) return VELORA_ERR_INVALID_ARG;
     if (ldx < D) return VELORA_ERR_INVALID_ARG;
     if (!elem_aligned(X, x_dtype) || !elem_aligned(v, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
     if (!ws || ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
     if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
-    if (N == 0) return VELORA_ERR_DEGENERATE_V;
     return launch_init_v(X, x_dtype, N, D, ldx, Dsub, v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
                     const float* v, void* Z, int z_dtype, int64_t ldz, void* stream)
 {
-    if (!X || !v || !Z) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
     if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (N == 0) return VELORA_OK;                    /* empty tensors may carry NULL pointers */
+    if (!X || !v || !Z) return VELORA_ERR_INVALID_ARG;
     if (ldx < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
     if (!elem_aligned(X, x_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
         return VELORA_ERR_ALIGNMENT;
-    if (N == 0) return VELORA_OK;
     return launch_compress(X, x_dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, static_cast<cudaStream_t>(stream));
 }
 
 int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
                        const float* v, void* Xhat, int x_dtype, int64_t ldxhat, void* stream)
 {
-    if (!Z || !v || !Xhat) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
     if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (N == 0) return VELORA_OK;
+    if (!Z || !v || !Xhat) return VELORA_ERR_INVALID_ARG;
     if (ldxhat < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
     if (!elem_aligned(Xhat, x_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
         return VELORA_ERR_ALIGNMENT;
-    if (N == 0) return VELORA_OK;
     return launch_reconstruct(Z, z_dtype, ldz, N, D, Dsub, v, Xhat, x_dtype, ldxhat,
                               static_cast<cudaStream_t>(stream));
 }
@@ -207,19 +229,21 @@ int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw
                           int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
                           void* ws, size_t ws_bytes, void* stream)
 {
-    (void)ws; (void)ws_bytes;
-    if (!X || !W || !v || !Y || !Z) return VELORA_ERR_INVALID_ARG;
     if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
     if (!valid_dtype(dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (N == 0) return VELORA_OK;
+    if (!X || !W || !v || !Y || !Z) return VELORA_ERR_INVALID_ARG;
     if (ldx < D || ldw < D || ldy < O || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
     if (!elem_aligned(X, dtype) || !elem_aligned(W, dtype) || !elem_aligned(Y, dtype) ||
         !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
         return VELORA_ERR_ALIGNMENT;
-    if (N == 0) return VELORA_OK;
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    rc = launch_linear_forward_tc(X, ldx, W, ldw, v, Y, ldy, Z, z_dtype, ldz, dtype, N, D, O, Dsub, s);
+    rc = launch_linear_forward_tc(X, ldx, W, ldw, v, Y, ldy, Z, z_dtype, ldz, dtype, N, D, O, Dsub,
+                                  static_cast<int*>(ws), s);
     if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     rc = launch_gemm_simt(X, dtype, ldx, 1, W, dtype, ldw, 1, Y, dtype, ldy, 0, N, O, D, s);
     if (rc != VELORA_OK) return rc;
@@ -253,9 +277,12 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
                                                    N, D, O, Dsub);
         if (ws_bytes < need) return VELORA_ERR_WORKSPACE;
     }
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (dX && N > 0) {
-        rc = launch_gemm_tc(GEMM_NN_K_MN, dY, lddy, W, ldw, dX, dtype, lddx, 0, N, D, O, dtype, s);
+        rc = launch_gemm_tc(GEMM_NN_K_MN, dY, lddy, W, ldw, dX, dtype, lddx, 0, N, D, O, dtype,
+                            static_cast<int*>(ws), s);
         if (rc == VELORA_ERR_UNSUPPORTED)
             rc = launch_gemm_simt(dY, dtype, lddy, 1, W, dtype, 1, ldw, dX, dtype, lddx, 0, N, D, O, s);
         if (rc != VELORA_OK) return rc;

@@ -1,23 +1,381 @@
+// Dense products of Algorithm 1 (arxiv 2405.17991) on the sm_100a tensor cores:
+//   Y = X W^T (forward), dX = dY W (input gradient), dW = dY^T Xhat (explicit weight gradient).
+//
+// One persistent, warp-specialised kernel: C[Mdim, Ndim] = A * B with bf16 operands and fp32
+// accumulation.  Output tile 128 x 256, K step 64.  Warp 0 feeds a 4-stage shared-memory ring with
+// TMA tile loads (128-byte swizzle); warp 1 issues tcgen05.mma (M = 128, N = 256, K = 16) into one of
+// two 256-column TMEM accumulators; warps 2..5 drain the other accumulator with tcgen05.ld, convert
+// and store, so the epilogue of a tile overlaps the main loop of the next.  Either operand may be
+// K-major (rows contiguous along K) or MN-major (rows contiguous along M or N): the latter is loaded
+// as 64 x 64 boxes and consumed through an MN-major matrix descriptor, so no transpose pass exists.
+// Ragged edges rely on TMA zero fill for loads and on predicated stores.
 #include "gemm_tc.cuh"
+#include "tc_common.cuh"
 
 namespace velora {
 
-int launch_gemm_tc(int, const void*, int64_t, const void*, int64_t, void*, int, int64_t, int,
-                   int64_t, int64_t, int64_t, int, cudaStream_t)
+using namespace tc;
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;              // 16 KB
+constexpr int B_BYTES = BN * BK * 2;              // 32 KB
+constexpr int SLAB_BYTES = 64 * BK * 2;           // one 64-wide MN-major slab: 64 k-rows x 128 bytes
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256;
+
+struct TileCoord {
+    int m0, n0;
+};
+
+// Tiles are walked in bands of 8 m-tiles so that CTAs running together share B tiles in L2.
+__device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles_n)
 {
-    return VELORA_ERR_UNSUPPORTED;
+    constexpr int BAND = 8;
+    const int per_band = BAND * tiles_n;
+    const int band = tile / per_band;
+    const int in_band = tile - band * per_band;
+    const int band_rows = (tiles_m - band * BAND < BAND) ? tiles_m - band * BAND : BAND;
+    const int tn = in_band / band_rows;
+    const int tm = band * BAND + (in_band - tn * band_rows);
+    return {tm * BM, tn * BN};
 }
 
-int launch_linear_forward_tc(const void*, int64_t, const void*, int64_t, const float*, void*, int64_t, void*, int,
-                             int64_t, int, int64_t, int64_t, int64_t, int, cudaStream_t)
+template <typename CT> struct Store32;
+template <> struct Store32<__nv_bfloat16> {
+    // 32 consecutive outputs of one row.
+    static __device__ __forceinline__ void run(__nv_bfloat16* p, const uint32_t (&r)[32], int valid, int beta)
+    {
+        if (valid >= 32) {
+            uint4* q = reinterpret_cast<uint4*>(p);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * i + e]);
+                if (beta) {
+                    const uint4 old = q[i];
+                    f[0] += bf16_lo(old.x); f[1] += bf16_hi(old.x);
+                    f[2] += bf16_lo(old.y); f[3] += bf16_hi(old.y);
+                    f[4] += bf16_lo(old.z); f[5] += bf16_hi(old.z);
+                    f[6] += bf16_lo(old.w); f[7] += bf16_hi(old.w);
+                }
+                uint4 o;
+                o.x = pack_bf16x2(f[0], f[1]);
+                o.y = pack_bf16x2(f[2], f[3]);
+                o.z = pack_bf16x2(f[4], f[5]);
+                o.w = pack_bf16x2(f[6], f[7]);
+                q[i] = o;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+                if (e < valid) {
+                    float f = __uint_as_float(r[e]);
+                    if (beta) f += __bfloat162float(p[e]);
+                    p[e] = __float2bfloat16_rn(f);
+                }
+        }
+    }
+};
+template <> struct Store32<float> {
+    static __device__ __forceinline__ void run(float* p, const uint32_t (&r)[32], int valid, int beta)
+    {
+        if (valid >= 32) {
+            float4* q = reinterpret_cast<float4*>(p);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float4 o = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                       __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                if (beta) {
+                    const float4 old = q[i];
+                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                q[i] = o;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+                if (e < valid) {
+                    float f = __uint_as_float(r[e]);
+                    if (beta) f += p[e];
+                    p[e] = f;
+                }
+        }
+    }
+};
+
+template <bool A_MN, bool B_MN, typename CT>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               CT* __restrict__ C, int64_t ldc, int beta, int Mdim, int Ndim, int Kdim,
+               int tiles_m, int tiles_n, int* __restrict__ status)
 {
-    return VELORA_ERR_UNSUPPORTED;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;               // swizzled tiles need 1024-byte alignment
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t sA = base;
+    const uint32_t sB = base + STAGES * A_BYTES;
+    uint8_t* tail = smem + STAGES * (A_BYTES + B_BYTES);
+    const uint32_t bars = base + STAGES * (A_BYTES + B_BYTES);
+    const uint32_t full = bars, empty = bars + 8 * STAGES;
+    const uint32_t tfull = bars + 16 * STAGES, tempty = tfull + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 40);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = tiles_m * tiles_n;
+    const int kblocks = (Kdim + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full + 8 * s, 1);
+            mbar_init(empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull + 8 * a, 1);
+            mbar_init(tempty + 8 * a, 4);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool failed = false;
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
+                const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+                    mbar_arrive_expect_tx(full + 8 * s, A_BYTES + B_BYTES);
+                    const int k0 = kb * BK;
+                    if (A_MN) {
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i)
+                            tma_load_2d(sA + s * A_BYTES + i * SLAB_BYTES, &tmA, full + 8 * s, tc0.m0 + 64 * i, k0);
+                    } else {
+                        tma_load_2d(sA + s * A_BYTES, &tmA, full + 8 * s, k0, tc0.m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i)
+                            tma_load_2d(sB + s * B_BYTES + i * SLAB_BYTES, &tmB, full + 8 * s, tc0.n0 + 64 * i, k0);
+                    } else {
+                        tma_load_2d(sB + s * B_BYTES, &tmB, full + 8 * s, k0, tc0.n0);
+                    }
+                }
+            }
+            if (failed) {
+                *abort_flag = 1;
+                // Let this CTA's own copies in flight land before shared memory is given up.
+                const uint32_t back = it < STAGES ? it : STAGES;
+                for (uint32_t j = 1; j <= back; ++j) {
+                    const uint32_t jt = it - j;
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full + 8 * (jt % STAGES), (jt / STAGES) & 1u))
+                        if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, A_MN, B_MN);
+            uint32_t it = 0, t = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x, ++t) {
+                const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
+                if (!mbar_wait(tempty + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(full + 8 * s, ph, abort_flag)) { failed = true; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = sA + s * A_BYTES, b_addr = sB + s * B_BYTES;
+#pragma unroll
+                    for (int j = 0; j < BK / 16; ++j) {
+                        // K-major: 16 elements of K = 32 bytes inside the swizzled 128-byte row.
+                        // MN-major: 16 k-rows of 128 bytes; 64-wide slabs are BK*128 bytes apart.
+                        const uint64_t da = A_MN ? umma_smem_desc(a_addr + j * 2048, SLAB_BYTES, 1024)
+                                                 : umma_smem_desc(a_addr + j * 32, 16, 1024);
+                        const uint64_t db = B_MN ? umma_smem_desc(b_addr + j * 2048, SLAB_BYTES, 1024)
+                                                 : umma_smem_desc(b_addr + j * 32, 16, 1024);
+                        umma_bf16(d_tmem, da, db, idesc, (kb | j) != 0);
+                    }
+                    umma_commit(empty + 8 * s);           // the stage is free once these MMAs have read it
+                }
+                if (failed) break;
+                umma_commit(tfull + 8 * acc);             // the accumulator is complete
+            }
+            if (failed) *abort_flag = 1;
+        }
+    } else {
+        // ------------------------------------------------ epilogue (4 warps, one TMEM lane quarter each)
+        const int quarter = warp & 3;
+        uint32_t t = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x, ++t) {
+            const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
+            const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
+            if (!mbar_wait(tfull + 8 * acc, aph, abort_flag)) { failed = true; break; }
+            tc_fence_after_sync();
+            const int row = tc0.m0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + acc * BN + (static_cast<uint32_t>(quarter * 32) << 16);
+            CT* crow = C + static_cast<int64_t>(row) * ldc + tc0.n0;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + c * 32, r);
+                tmem_ld_wait();
+                if (c == BN / 32 - 1) {                   // accumulator fully read: hand it back
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty + 8 * acc);
+                }
+                const int valid = Ndim - (tc0.n0 + c * 32);
+                if (row < Mdim && valid > 0) Store32<CT>::run(crow + c * 32, r, valid, beta);
+            }
+        }
+        if (failed) *abort_flag = 1;
+    }
+    if (failed && status) atomicExch(status, VELORA_ERR_TIMEOUT);
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+template <bool A_MN, bool B_MN, typename CT>
+int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t ldc, int beta,
+                  int Mdim, int Ndim, int Kdim, int* status, cudaStream_t stream)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
+    auto kern = gemm_tc_kernel<A_MN, B_MN, CT>;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(GEMM_SMEM)) != cudaSuccess)
+            return VELORA_ERR_CUDA;
+        configured[dev] = true;
+    }
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != VELORA_OK) return rc;
+    const int tiles_m = (Mdim + BM - 1) / BM, tiles_n = (Ndim + BN - 1) / BN;
+    const int64_t tiles = static_cast<int64_t>(tiles_m) * tiles_n;
+    const int grid = static_cast<int>(tiles < di.sm_count ? tiles : di.sm_count);
+    kern<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tb, static_cast<CT*>(C), ldc, beta, Mdim, Ndim, Kdim,
+                                                   tiles_m, tiles_n, status);
+    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+}
+
+}  // namespace
+
+int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
+                      int box_inner, int box_outer)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return VELORA_ERR_CUDA;
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(ld_elems) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? VELORA_OK : VELORA_ERR_CUDA;
+}
+
+bool tc_operand_ok(const void* p, int64_t ld_elems)
+{
+    return aligned16(p) && ld_elems % 8 == 0 && ld_elems * 2 < (static_cast<int64_t>(1) << 40);
+}
+
+int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
+                   void* C, int c_dtype, int64_t ldc, int beta,
+                   int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream)
+{
+    if (in_dtype != VELORA_BF16) return VELORA_ERR_UNSUPPORTED;
+    if (Mdim < 1 || Ndim < 1 || Kdim < 1) return VELORA_ERR_UNSUPPORTED;
+    if (Mdim > (1 << 30) || Ndim > (1 << 30) || Kdim > (1 << 30)) return VELORA_ERR_UNSUPPORTED;
+    if (!tc_operand_ok(A, lda) || !tc_operand_ok(B, ldb)) return VELORA_ERR_UNSUPPORTED;
+    if (!aligned16(C) || (ldc * static_cast<int64_t>(dtype_size(c_dtype))) % 16) return VELORA_ERR_UNSUPPORTED;
+    if ((static_cast<int64_t>((Mdim + BM - 1) / BM) * ((Ndim + BN - 1) / BN)) > (1 << 30)) return VELORA_ERR_UNSUPPORTED;
+
+    const bool a_mn = (kind == GEMM_TN_MN_MN);
+    const bool b_mn = (kind != GEMM_NT_K_K);
+    CUtensorMap ta, tb;
+    int rc;
+    // K-major operand: [rows = M or N][K], box 64 (K) x tile rows.  MN-major: [K][M or N], box 64 x 64.
+    rc = a_mn ? make_tmap_bf16_2d(&ta, A, Mdim, Kdim, lda, 64, BK) : make_tmap_bf16_2d(&ta, A, Kdim, Mdim, lda, BK, BM);
+    if (rc != VELORA_OK) return rc;
+    rc = b_mn ? make_tmap_bf16_2d(&tb, B, Ndim, Kdim, ldb, 64, BK) : make_tmap_bf16_2d(&tb, B, Kdim, Ndim, ldb, BK, BN);
+    if (rc != VELORA_OK) return rc;
+
+    const int m = static_cast<int>(Mdim), n = static_cast<int>(Ndim), k = static_cast<int>(Kdim);
+#define VELORA_GEMM_CASE(AMN, BMN)                                                                        \
+    return c_dtype == VELORA_BF16                                                                         \
+               ? launch_kernel<AMN, BMN, __nv_bfloat16>(ta, tb, C, ldc, beta, m, n, k, status, stream)    \
+               : launch_kernel<AMN, BMN, float>(ta, tb, C, ldc, beta, m, n, k, status, stream)
+    if (!a_mn && !b_mn) { VELORA_GEMM_CASE(false, false); }
+    if (!a_mn && b_mn) { VELORA_GEMM_CASE(false, true); }
+    VELORA_GEMM_CASE(true, true);
+#undef VELORA_GEMM_CASE
+}
+
+int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
+                             void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
+                             int dtype, int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream)
+{
+    int rc = launch_gemm_tc(GEMM_NT_K_K, X, ldx, W, ldw, Y, dtype, ldy, 0, N, O, D, dtype, status, stream);
+    if (rc != VELORA_OK) return rc;
+    return launch_compress(X, dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, stream);
 }
 
 size_t weight_grad_tc_workspace_bytes(int64_t, int64_t, int64_t, int) { return 0; }
 
 int launch_weight_grad_tc(const void*, int, int64_t, int64_t, int64_t, const void*, int, int64_t, const float*,
-                          int64_t, int, void*, int, int64_t, int, void*, size_t, cudaStream_t)
+                          int64_t, int, void*, int, int64_t, int, void*, size_t, int*, cudaStream_t)
 {
     return VELORA_ERR_UNSUPPORTED;
 }

@@ -12,22 +12,24 @@ enum GemmKind {
     GEMM_TN_MN_MN = 2   // dW = dY^T Xh: A[K, Mdim] contiguous in Mdim,   B[K, Ndim] contiguous in Ndim
 };
 
+// `status` (may be NULL) is a device word that a kernel sets to VELORA_ERR_TIMEOUT if one of its bounded
+// waits expires; nothing ever clears it but velora_workspace_init.
 // Returns VELORA_ERR_UNSUPPORTED (nothing launched) when the operands do not meet the tensor-core
 // path's requirements (bf16 data, 16-byte aligned rows); the caller then uses the CUDA-core GEMM.
 int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
                    void* C, int c_dtype, int64_t ldc, int beta,
-                   int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, cudaStream_t stream);
+                   int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream);
 
 // Y = X W^T with compress(X, v) computed from the same staged X tiles.
 int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
                              void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
-                             int dtype, int64_t N, int64_t D, int64_t O, int Dsub, cudaStream_t stream);
+                             int dtype, int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
 
 // Factored weight gradient: P = dY^T Z on tensor cores (split over tokens), dW = P (x) v.
 size_t weight_grad_tc_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub);
 int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
                           const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
                           void* dW, int dw_dtype, int64_t lddw, int beta,
-                          void* ws, size_t ws_bytes, cudaStream_t stream);
+                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream);
 
 }  // namespace velora

@@ -447,7 +447,7 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
                   float* v, void* ws, size_t ws_bytes, cudaStream_t stream)
 {
     if (ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
-    int* status = static_cast<int*>(ws);
+    int* status = static_cast<int*>(ws) + 1;             // word 1: degenerate-sum flag of this call
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
     const int M = static_cast<int>(ceil_div64(D, Dsub));
     const VecShape vs = vec_shape(Dsub);
