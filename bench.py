@@ -1,0 +1,425 @@
+"""Benchmark of the VeLoRA linear forward + backward path on B200.
+
+Workload (``config.workload``): the seven projections of one LLaMA-7B-shaped block
+(q/k/v/o 4096->4096, up/gate 4096->11008, down 11008->4096), a batch of 4 x 2048 = 8192 tokens,
+sub-token length 64, bf16 data with fp32 accumulation, seeded synthetic activations and gradients.
+One step = for every layer: velora_linear_forward (Y = X W^T and Z = compress(X, v)) followed by
+velora_linear_backward (dX = dY W and the factored weight gradient).  The metric is tokens per second
+through that fwd+bwd pass.  Every tensor set is several times larger than L2, so nothing is served
+from cache between steps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  ``--impl reference`` times the fp64 CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "velora_linear_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+CONFIG_INDEX = 5
+DSUB = 64
+CPU_SAMPLE_TOKENS = 4
+
+
+def peaks():
+    """Measured peaks of this machine's B200s if present, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _names(self, mask: int):
+        nv = self.nv
+        table = {
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake_slowdown": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        return [k for k, bit in table.items() if mask & bit]
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.reasons.update(self._names(int(mask)))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ------------------------------------------------------------------ multi-rank helpers (host logic)
+def aggregate_over_ranks(elapsed_ms_local: float, tokens_local: int, dist=None, device=None):
+    """MAX of the elapsed time and SUM of the tokens over all ranks (identity without a process group)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return elapsed_ms_local, tokens_local
+    import torch
+    t = torch.tensor([elapsed_ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([tokens_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
+def layer_flops(N, D, O, M):
+    """Algorithmic flops: the two dense products and the factored weight gradient."""
+    return {"fwd": 2.0 * N * D * O, "dx": 2.0 * N * D * O, "dw": 2.0 * N * O * M + O * D}
+
+
+# ------------------------------------------------------------------ CPU oracle leg
+def oracle_prepare(cfg, sample_tokens: int):
+    """Inputs of the oracle sample: the first ``sample_tokens`` tokens of every layer, widened to fp64."""
+    import oracle
+    import velora_inputs as vi
+    layers = []
+    for li, layer in enumerate(cfg.layers):
+        X = vi.make_X(cfg, li, N=sample_tokens).f64()
+        W = vi.make_W(cfg, li).f64()
+        dY = vi.make_dY(cfg, li, N=sample_tokens).f64()
+        v = oracle.init_v(X + 0.01, DSUB)
+        layers.append((X, W, dY, v, layer.D))
+    return layers
+
+
+def oracle_step(layers):
+    """One pass of the oracle, as it stands: forward product, compress, input gradient and the weight
+    gradient by its plain definition, for every layer."""
+    import oracle
+    for X, W, dY, v, D in layers:
+        oracle.linear_forward(X, W)
+        Z = oracle.compress(X, v)
+        oracle.input_grad(dY, W)
+        oracle.weight_grad(dY, Z, v, D)
+
+
+CPU_SAMPLE_TEXT = ("first %d tokens of each of the 7 layers: forward product, compress, input gradient, "
+                   "weight gradient by definition" % CPU_SAMPLE_TOKENS)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    import velora_inputs as vi
+    cfg = vi.CONFIGS[CONFIG_INDEX]
+    oracle.build()
+    layers = oracle_prepare(cfg, CPU_SAMPLE_TOKENS)
+    for _ in range(args.warmup):
+        oracle_step(layers)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(layers)
+    per_step = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = CPU_SAMPLE_TOKENS / per_step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": CPU_SAMPLE_TEXT},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": "config %d: %s, N=%d tokens, 7 projections (q,k,v,o 4096x4096; up,gate 4096x11008; "
+                        "down 11008x4096), Dsub=%d" % (cfg.index, cfg.name, cfg.N, DSUB),
+            "tokens": cfg.N, "Dsub": DSUB, "z_dtype": "f32", "dw": "factored",
+            "l2": "inputs larger than L2 (each step touches > 2 GB)"}
+
+
+# ------------------------------------------------------------------ GPU leg
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2405_17991_b200 as vl
+    import velora_inputs as vi
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    vl.lib()
+
+    cfg = vi.CONFIGS[CONFIG_INDEX]
+    N = cfg.N
+    pk = peaks()
+
+    # ---- inputs: generated once on the host (seeded), pinned, then resident in HBM
+    L = []
+    for li, layer in enumerate(cfg.layers):
+        hX = vi.make_X(cfg, li).torch("cpu").pin_memory()
+        hdY = vi.make_dY(cfg, li).torch("cpu").pin_memory()
+        W = vi.make_W(cfg, li).torch(dev)
+        X, dY = hX.to(dev), hdY.to(dev)
+        M = vl.num_subtokens(layer.D, DSUB)
+        v = vl.velora_init_v(X, DSUB)
+        L.append({
+            "name": layer.name, "D": layer.D, "O": layer.O, "M": M, "hX": hX, "hdY": hdY, "X": X, "dY": dY, "W": W,
+            "v": v, "Y": torch.empty((N, layer.O), dtype=torch.bfloat16, device=dev),
+            "Z": torch.empty((N, M), dtype=torch.float32, device=dev),
+            "dX": torch.empty((N, layer.D), dtype=torch.bfloat16, device=dev),
+            "dW": torch.empty((layer.O, layer.D), dtype=torch.bfloat16, device=dev),
+        })
+    ws_bytes = max(vl.velora_workspace_bytes(vl.OP_LINEAR_BACKWARD_FACTORED, N, l["D"], l["O"], DSUB) for l in L)
+    ws = vl.velora_workspace_alloc(ws_bytes, dev)
+
+    def step(events=None):
+        for l in L:
+            if events is not None:
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+            vl.velora_linear_forward(l["X"], l["W"], l["v"], Y=l["Y"], Z=l["Z"], ws=ws)
+            if events is not None:
+                e1.record()
+            vl.velora_linear_backward(l["dY"], l["W"], l["Z"], l["v"], dX=l["dX"], dW=l["dW"], ws=ws)
+            if events is not None:
+                e2.record()
+                events.append((l, e0, e1, e2))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = vl.velora_launch_count()
+    events = []
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start.record()
+        for _ in range(args.steps):
+            step(events)
+        end.record()
+        barrier()
+    elapsed_ms = start.elapsed_time(end)
+    launches = vl.velora_launch_count() - launches0
+    status = vl.velora_workspace_status(ws)
+    if status != 0:
+        raise RuntimeError("device status %d (%s) after the timed region" % (status, vl.velora_status_string(status)))
+    total_ms, total_tokens = aggregate_over_ranks(elapsed_ms, N * args.steps, dist if world > 1 else None, dev)
+    value = total_tokens / (total_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (the forward tensor-core GEMM), from the events of the timed region
+    fwd_ms = sum(e0.elapsed_time(e1) for (_, e0, e1, _) in events)
+    bwd_ms = sum(e1.elapsed_time(e2) for (_, _, e1, e2) in events)
+    fwd_flops = sum(layer_flops(N, l["D"], l["O"], l["M"])["fwd"] for (l, _, _, _) in events)
+    achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
+    peak = pk["bf16_tflops_sustained"]
+    roofline = {"kernel": "velora_linear_forward (tensor-core GEMM Y = X W^T with compress)", "bound": "tensor",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": "%s, sustained bf16 GEMM" % pk["source"], "traffic": None,
+                "launches": len(events), "avg_launch_ms": fwd_ms / max(len(events), 1),
+                "fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg), "clocks": clocks.summary(),
+        "gpu_launches": int(launches), "roofline": roofline,
+    }
+
+    if rank == 0:
+        line["kernels"] = kernel_table(vl, torch, L, N, ws, pk)
+
+    # ---- end to end: host buffers in, gradients out, through velora_linear_step_host
+    e2e_steps = max(1, min(args.steps, 5))
+    staging_bytes = max(vl.velora_host_step_staging_bytes(N, l["D"], l["O"], DSUB) for l in L)
+    staging = torch.empty(staging_bytes, dtype=torch.uint8, device=dev)
+    for l in L:
+        l["hdW"] = torch.empty((l["O"], l["D"]), dtype=torch.bfloat16).pin_memory()
+
+    def host_step():
+        for l in L:
+            vl.velora_linear_step_host(l["hX"], l["hdY"], l["W"], l["v"], staging, ws, hdW=l["hdW"])
+
+    host_step()
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for _ in range(e2e_steps):
+        host_step()
+    e2.record()
+    barrier()
+    e2e_ms, e2e_tokens = aggregate_over_ranks(s2.elapsed_time(e2), N * e2e_steps, dist if world > 1 else None, dev)
+    line["e2e"] = {
+        "value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+        "h2d_bytes_per_step": int(sum(N * (l["D"] + l["O"]) * 2 for l in L)),
+        "d2h_bytes_per_step": int(sum(l["O"] * l["D"] * 2 for l in L)),
+        "api": "velora_linear_step_host (pinned host X, dY in; dW out)",
+    }
+
+    if rank == 0:
+        import oracle
+        layers = oracle_prepare(cfg, CPU_SAMPLE_TOKENS)
+        reps, t0 = 0, time.perf_counter()
+        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+            oracle_step(layers)
+            reps += 1
+        t_cpu = (time.perf_counter() - t0) / reps
+        line["cpu_baseline"] = {
+            "value": CPU_SAMPLE_TOKENS / t_cpu, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": CPU_SAMPLE_TEXT + "; %d passes, %.2f s each" % (reps, t_cpu),
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def kernel_table(vl, torch, L, N, ws, pk):
+    """Per-kernel device times (CUDA events, inputs rotated so that every launch misses L2)."""
+    dev = L[0]["X"].device
+    by = {l["name"]: l for l in L}
+    out = []
+
+    def timed(fn_list, reps=5):
+        for f in fn_list:
+            f()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            for f in fn_list:
+                f()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (reps * len(fn_list))
+
+    def hbm(name, shape, ms, nbytes):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out.append({"kernel": name, "shape": shape, "us": ms * 1e3, "GB/s": gbs, "bound": "hbm",
+                    "frac_measured": gbs / pk["hbm_gbs"], "frac_nominal_8TBs": gbs / 8000.0})
+
+    def tensor(name, shape, ms, flops, nbytes=None):
+        tf = flops / (ms * 1e-3) / 1e12
+        row = {"kernel": name, "shape": shape, "us": ms * 1e3, "TFLOP/s": tf, "bound": "tensor",
+               "frac_measured_burst": tf / pk["bf16_tflops"]}
+        if nbytes is not None:                         # factored dW: HBM-bound, graded on bytes
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            ai = flops / nbytes
+            row.update({"bound": "hbm", "GB/s": gbs, "frac_measured": gbs / pk["hbm_gbs"],
+                        "roofline_TFLOP/s": min(pk["bf16_tflops"], ai * pk["hbm_gbs"] / 1e3)})
+        out.append(row)
+
+    # streaming kernels: the four 4096-wide inputs rotate (4 x 67 MB), the 11008-wide one is 180 MB alone
+    small = [by[n] for n in ("q", "k", "v", "o")]
+    big = by["down"]
+    for group, label in ((small, "N=%d D=4096" % N), ([big], "N=%d D=11008" % N)):
+        D, M = group[0]["D"], group[0]["M"]
+        ms = timed([(lambda l=l: vl.velora_compress(l["X"], l["v"], Z=l["Z"])) for l in group])
+        hbm("compress", label, ms, N * D * 2 + N * M * 4)
+        ms = timed([(lambda l=l: vl.velora_reconstruct(l["Z"], l["v"], D, Xhat=l["dX"])) for l in group])
+        hbm("reconstruct", label, ms, N * D * 2 + N * M * 4)
+        ms = timed([(lambda l=l: vl.velora_init_v(l["X"], DSUB, v=l["v"], ws=ws)) for l in group])
+        hbm("init_v (incl. one stream sync)", label, ms, N * D * 2)
+    # weight gradient, factored: rotate over layers of equal shape
+    for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
+        group = [by[n] for n in names]
+        l0 = group[0]
+        ms = timed([(lambda l=l: vl.velora_weight_grad(l["dY"], l["Z"], l["v"], l["D"], dW=l["dW"], ws=ws)) for l in group])
+        fl = layer_flops(N, l0["D"], l0["O"], l0["M"])["dw"]
+        tensor("weight_grad factored", "%dx%d -> dW[%d,%d]" % (N, l0["O"], l0["O"], l0["D"]), ms, fl,
+               N * l0["O"] * 2 + N * l0["M"] * 4 + l0["O"] * l0["D"] * 2)
+    # dense contractions
+    for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
+        group = [by[n] for n in names]
+        l0 = group[0]
+        fl = 2.0 * N * l0["D"] * l0["O"]
+        ms = timed([(lambda l=l: vl.velora_linear_forward(l["X"], l["W"], l["v"], Y=l["Y"], Z=l["Z"], ws=ws)) for l in group])
+        tensor("linear_forward (GEMM + compress)", "%dx%dx%d" % (N, l0["D"], l0["O"]), ms, fl)
+        ms = timed([(lambda l=l: vl.velora_linear_backward(l["dY"], l["W"], l["Z"], l["v"], dX=l["dX"], need_dW=False, ws=ws))
+                    for l in group])
+        tensor("input_grad GEMM dX = dY W", "%dx%dx%d" % (N, l0["O"], l0["D"]), ms, fl)
+    l0 = by["q"]
+    ws_ex = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_WEIGHT_GRAD_EXPLICIT, N, l0["D"], l0["O"], DSUB), dev)
+    ms = timed([(lambda l=l: vl.velora_weight_grad(l["dY"], l["Z"], l["v"], l["D"], dW=l["dW"], mode=vl.WG_EXPLICIT, ws=ws_ex))
+                for l in [by[n] for n in ("q", "k", "v", "o")]])
+    tensor("weight_grad explicit (reconstruct + GEMM dY^T Xhat)", "%dx%dx%d" % (l0["O"], N, l0["D"]), ms,
+           2.0 * N * l0["D"] * l0["O"])
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -80,6 +80,9 @@ typedef enum {
 /* Library version, major*10000 + minor*100 + patch. */
 int velora_version(void);
 
+/* Number of kernels this library has launched in the calling process so far (all devices). */
+unsigned long long velora_launch_count(void);
+
 /* Static, human-readable name of a status code. */
 const char* velora_status_string(int status);
 
@@ -171,6 +174,25 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
                            void* dX, int64_t lddx, void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
                            int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * One forward + backward of a VeLoRA linear (Algorithm 1, both functions) on data
+ * that lives in HOST memory (bf16, dense rows: ld = width).  On `stream`, in order:
+ * copies X[N, D] and dY[N, O] from the host into the device staging area, runs
+ * velora_linear_forward and velora_linear_backward (factored weight gradient,
+ * beta = 0, fp32 Z), and copies Y[N, O], dX[N, D] and dW[O, D] back to the host
+ * (each host output may be NULL to skip its copy).  Nothing is synchronised: the
+ * host buffers must stay valid until the stream has drained, and should be
+ * page-locked for the copies to be asynchronous.
+ * hX, hdY, hY, hdX, hdW: HOST pointers.  W[O, D] (ld = D) and v[Dsub]: DEVICE.
+ * staging: DEVICE memory of velora_host_step_staging_bytes(N, D, O, Dsub) bytes,
+ * 256-byte aligned.  ws: velora_workspace_bytes(VELORA_OP_LINEAR_BACKWARD_FACTORED, ...).
+ */
+size_t velora_host_step_staging_bytes(int64_t N, int64_t D, int64_t O, int Dsub);
+int velora_linear_step_host(const void* hX, const void* hdY, void* hY, void* hdX, void* hdW,
+                            const void* W, const float* v, void* staging, size_t staging_bytes,
+                            int64_t N, int64_t D, int64_t O, int Dsub,
+                            void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -29,6 +29,9 @@ SIGNATURES = {
     "velora_version": (_int, []),
     "velora_status_string": (ctypes.c_char_p, [_int]),
     "velora_workspace_bytes": (_sz, [_int, _i64, _i64, _i64, _int]),
+    "velora_launch_count": (ctypes.c_ulonglong, []),
+    "velora_host_step_staging_bytes": (_sz, [_i64, _i64, _i64, _int]),
+    "velora_linear_step_host": (_int, [_p, _p, _p, _p, _p, _p, _p, _p, _sz, _i64, _i64, _i64, _int, _p, _sz, _p]),
     "velora_workspace_init": (_int, [_p, _sz, _p]),
     "velora_workspace_status": (_int, [_p, _p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
@@ -248,3 +251,38 @@ def velora_linear_backward(dY: torch.Tensor, W: torch.Tensor, Z: torch.Tensor, v
                                       _stream(stream))
     _check(rc, "velora_linear_backward")
     return dX, dW
+
+
+def velora_launch_count() -> int:
+    return int(lib().velora_launch_count())
+
+
+def velora_host_step_staging_bytes(N: int, D: int, O: int, Dsub: int) -> int:
+    return int(lib().velora_host_step_staging_bytes(N, D, O, Dsub))
+
+
+def _host_ptr(t: Optional[torch.Tensor], shape, name: str) -> ctypes.c_void_p:
+    if t is None:
+        return ctypes.c_void_p(0)
+    if t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CPU bfloat16 tensor of shape %r" % (name, tuple(shape)))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def velora_linear_step_host(hX: torch.Tensor, hdY: torch.Tensor, W: torch.Tensor, v: torch.Tensor,
+                            staging: torch.Tensor, ws: torch.Tensor, hY: Optional[torch.Tensor] = None,
+                            hdX: Optional[torch.Tensor] = None, hdW: Optional[torch.Tensor] = None,
+                            stream=None) -> None:
+    """Forward + backward on host-resident (pinned) X and dY; results copied back to the given host tensors."""
+    N, D = hX.shape
+    O = W.shape[0]
+    Dsub = v.shape[0]
+    wp, ldw = _mat(W, "W")
+    if ldw != D:
+        raise ValueError("W must be dense")
+    rc = lib().velora_linear_step_host(
+        _host_ptr(hX, (N, D), "hX"), _host_ptr(hdY, (N, O), "hdY"), _host_ptr(hY, (N, O), "hY"),
+        _host_ptr(hdX, (N, D), "hdX"), _host_ptr(hdW, (O, D), "hdW"), wp, _vec(v),
+        ctypes.c_void_p(staging.data_ptr()), staging.numel(), N, D, O, Dsub,
+        ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_linear_step_host")

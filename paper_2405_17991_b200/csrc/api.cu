@@ -25,6 +25,14 @@ int device_info(DeviceInfo* out)
     return VELORA_OK;
 }
 
+static unsigned long long g_launches = 0;
+
+int after_launch()
+{
+    __atomic_add_fetch(&g_launches, 1ull, __ATOMIC_RELAXED);
+    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+}
+
 namespace {
 
 bool elem_aligned(const void* p, int dt)
@@ -116,6 +124,8 @@ using namespace velora;
 extern "C" {
 
 int velora_version(void) { return 100; }
+
+unsigned long long velora_launch_count(void) { return __atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
 
 int velora_workspace_init(void* ws, size_t ws_bytes, void* stream)
 {
@@ -290,6 +300,51 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
     if (dW)
         return weight_grad_impl(dY, dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub, dW, dw_dtype, lddw,
                                 beta, mode, ws, ws_bytes, s);
+    return VELORA_OK;
+}
+
+size_t velora_host_step_staging_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
+{
+    if (N < 0 || D < 1 || O < 1 || Dsub < 1 || Dsub > D) return 0;
+    const size_t n = static_cast<size_t>(N), d = static_cast<size_t>(D), o = static_cast<size_t>(O);
+    const size_t m = static_cast<size_t>(num_subtokens(D, Dsub));
+    return align256(n * d * 2) * 2 + align256(n * o * 2) * 2 + align256(o * d * 2) + align256(n * m * 4);
+}
+
+int velora_linear_step_host(const void* hX, const void* hdY, void* hY, void* hdX, void* hdW,
+                            const void* W, const float* v, void* staging, size_t staging_bytes,
+                            int64_t N, int64_t D, int64_t O, int Dsub,
+                            void* ws, size_t ws_bytes, void* stream)
+{
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (N == 0) return VELORA_OK;
+    if (!hX || !hdY || !W || !v || !staging) return VELORA_ERR_INVALID_ARG;
+    if (D % 8 || O % 8) return VELORA_ERR_UNSUPPORTED;          /* dense bf16 rows must be 16-byte multiples */
+    if (staging_bytes < velora_host_step_staging_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(staging) % 256) return VELORA_ERR_ALIGNMENT;
+    const size_t n = static_cast<size_t>(N), d = static_cast<size_t>(D), o = static_cast<size_t>(O);
+    const int64_t M = num_subtokens(D, Dsub);
+    char* p = static_cast<char*>(staging);
+    void* dXin = p;  p += align256(n * d * 2);
+    void* ddX = p;   p += align256(n * d * 2);
+    void* ddY = p;   p += align256(n * o * 2);
+    void* dYout = p; p += align256(n * o * 2);
+    void* ddW = p;   p += align256(o * d * 2);
+    void* dZ = p;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dXin, hX, n * d * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (cudaMemcpyAsync(ddY, hdY, n * o * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return VELORA_ERR_CUDA;
+    rc = velora_linear_forward(dXin, D, W, D, v, dYout, O, dZ, VELORA_F32, M, VELORA_BF16, N, D, O, Dsub,
+                               ws, ws_bytes, stream);
+    if (rc != VELORA_OK) return rc;
+    rc = velora_linear_backward(ddY, O, W, D, dZ, VELORA_F32, M, v, ddX, D, ddW, VELORA_BF16, D, 0,
+                                VELORA_WG_FACTORED, VELORA_BF16, N, D, O, Dsub, ws, ws_bytes, stream);
+    if (rc != VELORA_OK) return rc;
+    if (hY && cudaMemcpyAsync(hY, dYout, n * o * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (hdX && cudaMemcpyAsync(hdX, ddX, n * d * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (hdW && cudaMemcpyAsync(hdW, ddW, o * d * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VELORA_ERR_CUDA;
     return VELORA_OK;
 }
 

@@ -21,6 +21,9 @@ struct DeviceInfo {
 // Attributes of the current device (cached per device ordinal).
 int device_info(DeviceInfo* out);
 
+// Call right after every kernel launch: counts it and turns a launch error into a status.
+int after_launch();
+
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : 4; }

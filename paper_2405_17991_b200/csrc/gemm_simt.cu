@@ -94,7 +94,7 @@ int dispatch_c(const void* A, int64_t a_sm, int64_t a_sk, const void* B, int64_t
         gemm_simt_kernel<AT, BT, float><<<grid, THREADS, 0, stream>>>(
             static_cast<const AT*>(A), a_sm, a_sk, static_cast<const BT*>(B), b_sn, b_sk,
             static_cast<float*>(C), ldc, beta, Mdim, Ndim, Kdim);
-    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    return after_launch();
 }
 
 }  // namespace

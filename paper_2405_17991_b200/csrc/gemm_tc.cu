@@ -306,7 +306,7 @@ int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t
     const int grid = static_cast<int>(tiles < di.sm_count ? tiles : di.sm_count);
     kern<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tb, static_cast<CT*>(C), ldc, beta, Mdim, Ndim, Kdim,
                                                    tiles_m, tiles_n, status);
-    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    return after_launch();
 }
 
 }  // namespace

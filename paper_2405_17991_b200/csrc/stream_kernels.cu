@@ -414,7 +414,7 @@ int stream_grid(int64_t items, int per_thread, int* grid)
 
 int check_launch()
 {
-    return cudaGetLastError() == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    return after_launch();
 }
 
 // Largest number of rows one vector launch may take so that item counts stay below 2^30.
