@@ -120,6 +120,28 @@ int velora_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
                   float* v, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * velora_init_v for callers that have no device memory to lend.  The paper has no counterpart: it is
+ * the same operation and the same kernels as velora_init_v, but the partial sums go to a fixed array
+ * inside the library instead of a caller-provided workspace.  It exists for code that runs where
+ * allocating is not an option: a plugin handed only its input and output buffers by a host framework
+ * that owns the allocator, a real-time loop that must not touch the driver's allocator once started,
+ * or start-up code that runs before the application's memory pool exists.  The call itself allocates
+ * and frees nothing, on the host or on the device.
+ *   - Limit: Dsub <= VELORA_INIT_V_STATIC_MAX_DSUB, else VELORA_ERR_UNSUPPORTED (use velora_init_v).
+ *   - Cost: the array (about 1.2 MB) is part of the library image, so every GPU on which the library
+ *     is used keeps it until the process ends.
+ *   - The first call on each device looks up the array's device address (once, cached); make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call overwrites what it reads, so calls need
+ *     no clearing between them, but two calls whose work overlaps on the GPU (different streams or
+ *     threads) race on it: serialise them.  Like velora_init_v it synchronises `stream` once.
+ * Arguments, results and errors otherwise as velora_init_v.
+ */
+#define VELORA_INIT_V_STATIC_MAX_DSUB 256
+int velora_init_v_static(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                         float* v, void* stream);
+
+/*
  * compress (Section 3.1, Eq. 1):  Z[n, m] = sum_j X[n, m*Dsub + j] * v[j].
  * X: [N, D] bf16 or f32.  v: fp32 [Dsub].  Z: [N, M] f32 or bf16, ldz >= M.
  * Products and sums are formed in fp32.

@@ -7,7 +7,7 @@ arguments.  Build the library with ``python -m paper_2405_17991_b200.build``.
 from .binding import (  # noqa: F401
     BF16, F32, LIB_PATH, OP_INIT_V, OP_LINEAR_BACKWARD_EXPLICIT, OP_LINEAR_BACKWARD_FACTORED,
     OP_LINEAR_FORWARD, OP_WEIGHT_GRAD_EXPLICIT, OP_WEIGHT_GRAD_FACTORED, SIGNATURES, WG_EXPLICIT,
-    WG_FACTORED, VeloraError, lib, num_subtokens, velora_compress, velora_init_v,
+    WG_FACTORED, VeloraError, lib, num_subtokens, velora_compress, velora_init_v, velora_init_v_static,
     velora_linear_backward, velora_linear_forward, velora_reconstruct, velora_status_string,
     velora_version, velora_weight_grad, velora_workspace_alloc, velora_workspace_bytes,
     velora_workspace_init, velora_workspace_status, velora_launch_count,

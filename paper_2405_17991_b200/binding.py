@@ -35,6 +35,7 @@ SIGNATURES = {
     "velora_workspace_init": (_int, [_p, _sz, _p]),
     "velora_workspace_status": (_int, [_p, _p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
+    "velora_init_v_static": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_reconstruct": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_weight_grad": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _p, _i64, _int,
@@ -155,6 +156,19 @@ def velora_init_v(X: torch.Tensor, Dsub: int, v: Optional[torch.Tensor] = None,
     rc = lib().velora_init_v(xp, _dt(X), N, D, ldx, Dsub, _vec(v), ctypes.c_void_p(ws.data_ptr()), ws.numel(),
                              _stream(stream))
     _check(rc, "velora_init_v")
+    return v
+
+
+def velora_init_v_static(X: torch.Tensor, Dsub: int, v: torch.Tensor, stream=None) -> torch.Tensor:
+    """velora_init_v through the library's built-in scratch: no workspace, nothing allocated by the call.
+
+    ``v`` must be supplied by the caller (this wrapper allocates nothing either).  Dsub is limited to
+    256; calls on one device must not overlap on the GPU, since they share the scratch array.
+    """
+    xp, ldx = _mat(X, "X")
+    N, D = X.shape
+    rc = lib().velora_init_v_static(xp, _dt(X), N, D, ldx, Dsub, _vec(v), _stream(stream))
+    _check(rc, "velora_init_v_static")
     return v
 
 

@@ -592,3 +592,55 @@ int launch_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int6
 }
 
 }  // namespace velora
+
+// ------------------------------------------------------------------ velora_init_v without a workspace
+// Scratch for velora_init_v_static: the status header plus one row of partial sums per CTA, for
+// sub-tokens of up to VELORA_INIT_V_STATIC_MAX_DSUB elements.  It is part of the loaded module, so
+// every GPU that loads the library carries these ~1.2 MB until the process exits.
+namespace velora {
+namespace {
+constexpr size_t kStaticScratchBytes =
+    kStatusBytes + static_cast<size_t>(kInitVMaxCtas) * VELORA_INIT_V_STATIC_MAX_DSUB * sizeof(float);
+static __device__ __align__(256) unsigned char g_init_v_scratch[kStaticScratchBytes];
+
+// Device address of g_init_v_scratch on the current device.  In host code the array's name is only a
+// handle for the runtime, never a pointer a kernel may use; the real address is asked for once per
+// device, with that device current, and remembered.
+int static_scratch_address(void** out)
+{
+    static void* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return VELORA_ERR_UNSUPPORTED;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_init_v_scratch) != cudaSuccess || !p) return VELORA_ERR_CUDA;
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return VELORA_OK;
+}
+}  // namespace
+}  // namespace velora
+
+extern "C" int velora_init_v_static(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                                    float* v, void* stream)
+{
+    using namespace velora;
+    if (N < 0 || D < 1 || Dsub < 1 || Dsub > D) return VELORA_ERR_INVALID_ARG;
+    if (Dsub > VELORA_INIT_V_STATIC_MAX_DSUB) return VELORA_ERR_UNSUPPORTED;   // beyond the built-in scratch
+    if (D > (1 << 30) || N > (static_cast<int64_t>(1) << 40)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (N == 0) return VELORA_ERR_DEGENERATE_V;
+    if (!X || !v) return VELORA_ERR_INVALID_ARG;
+    if (ldx < D) return VELORA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(X) % dtype_size(x_dtype) || reinterpret_cast<uintptr_t>(v) % sizeof(float))
+        return VELORA_ERR_ALIGNMENT;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != VELORA_OK) return rc;
+    // Every partial-sum row that is read was written by this call, and the result word is rewritten
+    // by every call, so nothing in the shared scratch has to be cleared first.
+    return launch_init_v(X, x_dtype, N, D, ldx, Dsub, v, scratch, kStaticScratchBytes,
+                         static_cast<cudaStream_t>(stream));
+}
