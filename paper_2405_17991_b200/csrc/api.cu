@@ -84,7 +84,7 @@ int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t
         float* P = reinterpret_cast<float*>(body);
         rc = launch_gemm_simt(dY, dy_dtype, 1, lddy, Z, z_dtype, 1, ldz, P, VELORA_F32, M, 0, O, M, N, stream);
         if (rc != VELORA_OK) return rc;
-        return launch_expand_p(P, M, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
+        return launch_expand_p(P, 1, 0, M, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
     }
     // Explicit: Xhat into the workspace in dY's storage type, then dW = dY^T Xhat.
     if (ws_bytes < xhat_bytes(N, D)) return VELORA_ERR_WORKSPACE;

@@ -46,9 +46,10 @@ int launch_gemm_simt(const void* A, int a_dtype, int64_t a_sm, int64_t a_sk,
                      void* C, int c_dtype, int64_t ldc, int beta,
                      int64_t Mdim, int64_t Ndim, int64_t Kdim, cudaStream_t stream);
 
-// dW[o, m*Dsub + j] = beta*dW + P[o, m] * v[j] with P[O, M] fp32 (expansion after a CUDA-core P = dY^T Z).
-int launch_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
-                    void* dW, int dw_dtype, int64_t lddw, int beta, cudaStream_t stream);
+// dW[o, m*Dsub + j] = beta*dW + (sum over `splits` partial P[s][o][m], fp32) * v[j].
+int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ldp, const float* v,
+                    int64_t O, int64_t D, int Dsub, void* dW, int dw_dtype, int64_t lddw, int beta,
+                    cudaStream_t stream);
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }

@@ -372,12 +372,4 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
     return launch_compress(X, dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, stream);
 }
 
-size_t weight_grad_tc_workspace_bytes(int64_t, int64_t, int64_t, int) { return 0; }
-
-int launch_weight_grad_tc(const void*, int, int64_t, int64_t, int64_t, const void*, int, int64_t, const float*,
-                          int64_t, int, void*, int, int64_t, int, void*, size_t, int*, cudaStream_t)
-{
-    return VELORA_ERR_UNSUPPORTED;
-}
-
 }  // namespace velora

@@ -1,6 +1,8 @@
 // Tensor-core (tcgen05 / TMA / TMEM) kernels of the VeLoRA path.
 #pragma once
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace velora {
@@ -19,6 +21,12 @@ enum GemmKind {
 int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
                    void* C, int c_dtype, int64_t ldc, int beta,
                    int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream);
+
+// Tensor map of a row-major bf16 matrix: `inner` contiguous elements per row, `outer` rows, row pitch
+// ld_elems; 128-byte swizzle, zero fill outside the matrix.  (gemm_tc.cu)
+int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
+                      int box_inner, int box_outer);
+bool tc_operand_ok(const void* p, int64_t ld_elems);
 
 // Y = X W^T with compress(X, v) computed from the same staged X tiles.
 int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,

@@ -355,11 +355,14 @@ reconstruct_elem_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D,
     }
 }
 
-// P[O, M] fp32 expanded to dW[o, m*Dsub + j] = beta*dW + P[o, m] v[j].
+// Expansion of the factored weight gradient (Section 3.2's rank-1 form, per sub-token):
+//   dW[o, m*Dsub + j] = beta*dW[o, m*Dsub + j] + (sum_s P[s][o][m]) * v[j]
+// P holds `splits` partial products dY^T Z over disjoint token ranges, summed here in a fixed order.
 template <typename WT>
 __global__ void __launch_bounds__(kStreamThreads)
-expand_p_kernel(const float* __restrict__ P, int64_t ldp, const float* __restrict__ v, int64_t O, int D, int Dsub,
-                WT* __restrict__ dW, int64_t lddw, int beta)
+expand_p_elem_kernel(const float* __restrict__ P, int splits, int64_t split_stride, int64_t ldp,
+                     const float* __restrict__ v, int64_t O, int D, int Dsub,
+                     WT* __restrict__ dW, int64_t lddw, int beta)
 {
     const int64_t total = O * D;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
@@ -368,9 +371,104 @@ expand_p_kernel(const float* __restrict__ P, int64_t ldp, const float* __restric
         const int d = static_cast<int>(idx - o * D);
         const int m = d / Dsub;
         const int j = d - m * Dsub;
-        float r = __ldg(P + o * ldp + m) * __ldg(v + j);
+        float p = 0.f;
+        for (int s = 0; s < splits; ++s) p += __ldg(P + s * split_stride + o * ldp + m);
+        float r = p * __ldg(v + j);
         if (beta) r += Elem<WT>::load(dW + o * lddw + d);
         Elem<WT>::store(dW + o * lddw + d, r);
+    }
+}
+
+template <typename WT> struct Chunk8;
+template <> struct Chunk8<__nv_bfloat16> {
+    static __device__ __forceinline__ void store(__nv_bfloat16* row, int col, float (&y)[8], int beta)
+    {
+        uint4* p = reinterpret_cast<uint4*>(row + col);
+        if (beta) {
+            const uint4 old = *p;
+            y[0] += bf16_lo(old.x); y[1] += bf16_hi(old.x);
+            y[2] += bf16_lo(old.y); y[3] += bf16_hi(old.y);
+            y[4] += bf16_lo(old.z); y[5] += bf16_hi(old.z);
+            y[6] += bf16_lo(old.w); y[7] += bf16_hi(old.w);
+        }
+        uint4 o;
+        o.x = pack_bf16x2(y[0], y[1]);
+        o.y = pack_bf16x2(y[2], y[3]);
+        o.z = pack_bf16x2(y[4], y[5]);
+        o.w = pack_bf16x2(y[6], y[7]);
+        __stcs(p, o);
+    }
+};
+template <> struct Chunk8<float> {
+    static __device__ __forceinline__ void store(float* row, int col, float (&y)[8], int beta)
+    {
+        float4* p = reinterpret_cast<float4*>(row + col);
+        if (beta) {
+            const float4 a = p[0], b = p[1];
+            y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
+            y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
+        }
+        __stcs(p, make_float4(y[0], y[1], y[2], y[3]));
+        __stcs(p + 1, make_float4(y[4], y[5], y[6], y[7]));
+    }
+};
+
+// Vector form: same item walk as reconstruct, rows are output rows o.
+template <int LPS, int CH, int U, typename WT>
+__global__ void __launch_bounds__(kStreamThreads)
+expand_p_vec_kernel(const float* __restrict__ P, int splits, int64_t split_stride, int64_t ldp,
+                    const float* __restrict__ v, int64_t O, int D, int M,
+                    WT* __restrict__ dW, int64_t lddw, int beta)
+{
+    constexpr int L = LPS * CH;
+    const int q = threadIdx.x & (LPS - 1);
+    float vr[CH][8];
+#pragma unroll
+    for (int i = 0; i < CH; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
+
+    ItemWalk w;
+    w.init(M * LPS);
+    while (w.row < O) {
+        float p[U];
+        int64_t rows[U];
+        int ms[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            rows[u] = w.row;
+            ms[u] = w.pos / LPS;
+            p[u] = 0.f;
+            if (w.row < O) {
+                const float* pp = P + w.row * ldp + ms[u];
+                for (int s = 0; s < splits; ++s) p[u] += __ldg(pp + s * split_stride);
+            }
+            w.advance();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (rows[u] < O) {
+                WT* row = dW + rows[u] * lddw;
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const int col = (ms[u] * L + q + LPS * i) * 8;
+                    float y[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) y[e] = p[u] * vr[i][e];
+                    if (col + 8 <= D) {
+                        Chunk8<WT>::store(row, col, y, beta);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (col + e < D) {
+                                float r = y[e];
+                                if (beta) r += Elem<WT>::load(row + col + e);
+                                Elem<WT>::store(row + col + e, r);
+                            }
+                    }
+                }
+            }
+        }
     }
 }
 
@@ -576,18 +674,37 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
     return check_launch();
 }
 
-int launch_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
-                    void* dW, int dw_dtype, int64_t lddw, int beta, cudaStream_t stream)
+int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ldp, const float* v,
+                    int64_t O, int64_t D, int Dsub, void* dW, int dw_dtype, int64_t lddw, int beta,
+                    cudaStream_t stream)
 {
+    const int M = static_cast<int>(ceil_div64(D, Dsub));
+    const VecShape vs = vec_shape(Dsub);
+    const bool rows16 = aligned16(dW) && (lddw * static_cast<int64_t>(dtype_size(dw_dtype))) % 16 == 0;
+    if (vs.ok && rows16 && O <= max_rows_per_launch(M * vs.lps)) {
+        int grid = 0;
+        int rc = stream_grid(O * M * vs.lps, vs.u, &grid);
+        if (rc != VELORA_OK) return rc;
+#define CALL_EXPAND(LPS, CH, U)                                                                            \
+        if (dw_dtype == VELORA_BF16)                                                                       \
+            expand_p_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(           \
+                P, splits, split_stride, ldp, v, O, static_cast<int>(D), M, static_cast<__nv_bfloat16*>(dW), lddw, beta); \
+        else                                                                                               \
+            expand_p_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(                   \
+                P, splits, split_stride, ldp, v, O, static_cast<int>(D), M, static_cast<float*>(dW), lddw, beta)
+        VELORA_DISPATCH_VEC(vs, CALL_EXPAND)
+#undef CALL_EXPAND
+        return check_launch();
+    }
     int grid = 0;
     int rc = stream_grid(O * D, 4, &grid);
     if (rc != VELORA_OK) return rc;
     if (dw_dtype == VELORA_BF16)
-        expand_p_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(
-            P, ldp, v, O, static_cast<int>(D), Dsub, static_cast<__nv_bfloat16*>(dW), lddw, beta);
+        expand_p_elem_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(
+            P, splits, split_stride, ldp, v, O, static_cast<int>(D), Dsub, static_cast<__nv_bfloat16*>(dW), lddw, beta);
     else
-        expand_p_kernel<float><<<grid, kStreamThreads, 0, stream>>>(
-            P, ldp, v, O, static_cast<int>(D), Dsub, static_cast<float*>(dW), lddw, beta);
+        expand_p_elem_kernel<float><<<grid, kStreamThreads, 0, stream>>>(
+            P, splits, split_stride, ldp, v, O, static_cast<int>(D), Dsub, static_cast<float*>(dW), lddw, beta);
     return check_launch();
 }
 

@@ -1,0 +1,292 @@
+// Factored weight gradient on the sm_100a tensor cores (arxiv 2405.17991, Algorithm 1 backward with
+// the rank-1 identity of Section 3.2 applied per sub-token):
+//     P[o, m] = sum_n dY[n, o] * Z[n, m],      dW[o, m*Dsub + j] = beta*dW + P[o, m] * v[j].
+// The reconstructed input is never formed.  The work is bound by HBM traffic (read dY once, write dW
+// once); the contraction over tokens is small next to it and runs on tcgen05 so that it hides under
+// the dY stream.
+//
+// Three launches:
+//   1. z_to_bf16_kernel   Z (fp32 or bf16, any pitch) -> Zb[N, pitch] bf16, pitch = round_up(M, 64),
+//                         zero padded, so that TMA can fetch 64-wide MN-major slabs.
+//   2. wg_partial_kernel  grid (O/128, splits): CTA (t, s) multiplies dY[:, 128t : 128t+128]^T with Zb
+//                         over its share of the tokens.  Both operands are MN-major (tokens are the K
+//                         dimension and rows of dY / Zb are tokens): 64 x 64 TMA boxes, MN-major
+//                         matrix descriptors, no transpose.  fp32 accumulator in TMEM, written as a
+//                         partial product P[s][o][m].
+//   3. expand_p kernel    sums the partials in fixed order and streams dW = P (x) v over all SMs.
+// Splitting the token range keeps every SM pulling on dY; summing partials in a fixed order keeps the
+// result run-to-run identical.
+#include "gemm_tc.cuh"
+#include "tc_common.cuh"
+
+namespace velora {
+
+using namespace tc;
+
+namespace {
+
+constexpr int WG_BM = 128, WG_BK = 64, WG_STAGES = 4;
+constexpr int WG_A_BYTES = WG_BM * WG_BK * 2;         // 16 KB: two 64-wide slabs of dY^T
+constexpr int WG_SLAB = 64 * WG_BK * 2;               // 8 KB
+constexpr int WG_THREADS = 192;
+constexpr int WG_MAX_SPLITS = 8;
+constexpr int WG_MAX_M = 256;
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+template <typename ZT>
+__global__ void __launch_bounds__(256)
+z_to_bf16_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int M, int pitch, uint4* __restrict__ Zb)
+{
+    const int chunks = pitch / 8;
+    const int64_t total = N * chunks;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
+        const int64_t n = idx / chunks;
+        const int c0 = static_cast<int>(idx - n * chunks) * 8;
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = (c0 + e < M) ? Elem<ZT>::load(Z + n * ldz + c0 + e) : 0.f;
+        uint4 o;
+        o.x = pack_bf16x2(f[0], f[1]);
+        o.y = pack_bf16x2(f[2], f[3]);
+        o.z = pack_bf16x2(f[4], f[5]);
+        o.w = pack_bf16x2(f[6], f[7]);
+        Zb[idx] = o;
+    }
+}
+
+__global__ void __launch_bounds__(WG_THREADS, 2)
+wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmZ,
+                  float* __restrict__ partials, int O, int n_slabs, int npad, int tmem_cols,
+                  int kblocks, int kb_per_split, int64_t split_stride, int ldp, int* __restrict__ status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const int stage_bytes = WG_A_BYTES + n_slabs * WG_SLAB;
+    uint8_t* tail = smem + WG_STAGES * stage_bytes;
+    const uint32_t bars = base + WG_STAGES * stage_bytes;
+    const uint32_t full = bars, empty = bars + 8 * WG_STAGES, tfull = bars + 16 * WG_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * WG_STAGES + 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * WG_STAGES + 24);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int o0 = blockIdx.x * WG_BM;
+    const int split = blockIdx.y;
+    const int kb0 = split * kb_per_split;
+    const int kb1 = (kb0 + kb_per_split < kblocks) ? kb0 + kb_per_split : kblocks;
+    const int nkb = kb1 - kb0;                               // >= 1 by construction on the host
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < WG_STAGES; ++s) {
+            mbar_init(full + 8 * s, 1);
+            mbar_init(empty + 8 * s, 1);
+        }
+        mbar_init(tfull, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmY);
+        prefetch_tensormap(&tmZ);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), static_cast<uint32_t>(tmem_cols));
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool failed = false;
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (; it < nkb; ++it) {
+                const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
+                if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+                mbar_arrive_expect_tx(full + 8 * s, static_cast<uint32_t>(stage_bytes));
+                const int k0 = (kb0 + it) * WG_BK;
+                const uint32_t a_dst = base + s * stage_bytes;
+                tma_load_2d(a_dst, &tmY, full + 8 * s, o0, k0);
+                tma_load_2d(a_dst + WG_SLAB, &tmY, full + 8 * s, o0 + 64, k0);
+                for (int i = 0; i < n_slabs; ++i)
+                    tma_load_2d(a_dst + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * s, 64 * i, k0);
+            }
+            if (failed) {
+                *abort_flag = 1;
+                const int back = it < WG_STAGES ? it : WG_STAGES;   // copies of this CTA still in flight
+                for (int j = 1; j <= back; ++j) {
+                    const int jt = it - j;
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full + 8 * (jt % WG_STAGES), (jt / WG_STAGES) & 1u))
+                        if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(WG_BM, npad, true, true);
+            for (int it = 0; it < nkb; ++it) {
+                const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
+                if (!mbar_wait(full + 8 * s, ph, abort_flag)) { failed = true; break; }
+                tc_fence_after_sync();
+                const uint32_t a_addr = base + s * stage_bytes, b_addr = a_addr + WG_A_BYTES;
+#pragma unroll
+                for (int j = 0; j < WG_BK / 16; ++j) {
+                    const uint64_t da = umma_smem_desc(a_addr + j * 2048, WG_SLAB, 1024);
+                    const uint64_t db = umma_smem_desc(b_addr + j * 2048, WG_SLAB, 1024);
+                    umma_bf16(tmem_base, da, db, idesc, (it | j) != 0);
+                }
+                umma_commit(empty + 8 * s);
+            }
+            if (!failed) umma_commit(tfull);
+            else *abort_flag = 1;
+        }
+    } else {
+        const int quarter = warp & 3;
+        if (!mbar_wait(tfull, 0u, abort_flag)) {
+            failed = true;
+            *abort_flag = 1;
+        } else {
+            tc_fence_after_sync();
+            const int o = o0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            float* prow = partials + split * split_stride + static_cast<int64_t>(o) * ldp;
+            for (int c = 0; c * 32 < npad; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + c * 32, r);
+                tmem_ld_wait();
+                if (o < O) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (c * 32 + 4 * i < npad)                 // npad is a multiple of 16
+                            *reinterpret_cast<float4*>(prow + c * 32 + 4 * i) =
+                                make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                            __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                }
+            }
+        }
+    }
+    if (failed && status) atomicExch(status, VELORA_ERR_TIMEOUT);
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, static_cast<uint32_t>(tmem_cols));
+    }
+}
+
+struct WgPlan {
+    bool ok;
+    int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o;
+    size_t zb_bytes, part_bytes, smem;
+};
+
+WgPlan make_plan(int64_t N, int64_t D, int64_t O, int Dsub, int sm_count)
+{
+    WgPlan p{};
+    const int64_t M = ceil_div64(D, Dsub);
+    if (M > WG_MAX_M || N < 1 || N > (1 << 30) || O > (1 << 30)) return p;
+    p.M = static_cast<int>(M);
+    p.npad = static_cast<int>(round_up(M, 16));
+    p.pitch = static_cast<int>(round_up(M, 64));
+    p.n_slabs = p.pitch / 64;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.npad) p.tmem_cols *= 2;
+    p.kblocks = static_cast<int>(ceil_div64(N, WG_BK));
+    p.tiles_o = static_cast<int>(ceil_div64(O, WG_BM));
+    p.smem = 1024 + static_cast<size_t>(WG_STAGES) * (WG_A_BYTES + p.n_slabs * WG_SLAB) + 256;
+    const int64_t slots = static_cast<int64_t>(sm_count) * (2 * (p.smem + 1024) <= 228 * 1024 ? 2 : 1);
+    // Pick the split count that fills whole waves of SMs best; ties go to fewer splits (fewer partials).
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= WG_MAX_SPLITS && s <= p.kblocks; ++s) {
+        const int64_t ctas = static_cast<int64_t>(p.tiles_o) * s;
+        const int64_t waves = ceil_div64(ctas, slots);
+        const double eff = static_cast<double>(ctas) / static_cast<double>(waves * slots) - 0.01 * s;
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
+    }
+    p.kb_per_split = static_cast<int>(ceil_div64(p.kblocks, best));
+    p.splits = static_cast<int>(ceil_div64(p.kblocks, p.kb_per_split));
+    p.zb_bytes = static_cast<size_t>(round_up(static_cast<int64_t>(N) * p.pitch * 2, 256));
+    p.part_bytes = static_cast<size_t>(WG_MAX_SPLITS) * static_cast<size_t>(O) * p.npad * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+}  // namespace
+
+size_t weight_grad_tc_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
+{
+    const WgPlan p = make_plan(N > 0 ? N : 1, D, O, Dsub, 148);
+    if (!p.ok) return 0;
+    return p.zb_bytes + static_cast<size_t>(round_up(static_cast<int64_t>(p.part_bytes), 256));
+}
+
+int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                          const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                          void* dW, int dw_dtype, int64_t lddw, int beta,
+                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream)
+{
+    if (dy_dtype != VELORA_BF16 || N < 1) return VELORA_ERR_UNSUPPORTED;
+    if (!tc_operand_ok(dY, lddy)) return VELORA_ERR_UNSUPPORTED;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != VELORA_OK) return rc;
+    const WgPlan p = make_plan(N, D, O, Dsub, di.sm_count);
+    if (!p.ok) return VELORA_ERR_UNSUPPORTED;
+    if (ws_bytes < weight_grad_tc_workspace_bytes(N, D, O, Dsub) || !aligned16(ws)) return VELORA_ERR_WORKSPACE;
+    if (p.smem > static_cast<size_t>(di.smem_optin)) return VELORA_ERR_UNSUPPORTED;
+
+    uint4* Zb = static_cast<uint4*>(ws);
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + p.zb_bytes);
+
+    // 1. Z -> bf16, padded to whole 64-wide slabs
+    {
+        const int64_t items = N * (p.pitch / 8);
+        int64_t grid = ceil_div64(items, 256);
+        const int64_t cap = static_cast<int64_t>(di.sm_count) * 8;
+        if (grid > cap) grid = cap;
+        if (z_dtype == VELORA_F32)
+            z_to_bf16_kernel<float><<<static_cast<int>(grid), 256, 0, stream>>>(
+                static_cast<const float*>(Z), ldz, N, p.M, p.pitch, Zb);
+        else
+            z_to_bf16_kernel<__nv_bfloat16><<<static_cast<int>(grid), 256, 0, stream>>>(
+                static_cast<const __nv_bfloat16*>(Z), ldz, N, p.M, p.pitch, Zb);
+        rc = after_launch();
+        if (rc != VELORA_OK) return rc;
+    }
+    // 2. partial products on the tensor cores
+    {
+        CUtensorMap tmY, tmZ;
+        rc = make_tmap_bf16_2d(&tmY, dY, O, N, lddy, 64, WG_BK);
+        if (rc != VELORA_OK) return rc;
+        rc = make_tmap_bf16_2d(&tmZ, Zb, p.pitch, N, p.pitch, 64, WG_BK);
+        if (rc != VELORA_OK) return rc;
+        static bool configured[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(wg_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     di.smem_optin) != cudaSuccess)
+                return VELORA_ERR_CUDA;
+            configured[dev] = true;
+        }
+        const int64_t split_stride = static_cast<int64_t>(O) * p.npad;
+        dim3 grid(static_cast<unsigned>(p.tiles_o), static_cast<unsigned>(p.splits));
+        wg_partial_kernel<<<grid, WG_THREADS, p.smem, stream>>>(tmY, tmZ, partials, static_cast<int>(O), p.n_slabs,
+                                                               p.npad, p.tmem_cols, p.kblocks, p.kb_per_split,
+                                                               split_stride, p.npad, status);
+        rc = after_launch();
+        if (rc != VELORA_OK) return rc;
+    }
+    // 3. dW = (sum of partials) (x) v
+    return launch_expand_p(partials, p.splits, static_cast<int64_t>(O) * p.npad, p.npad, v, O, D, Dsub,
+                           dW, dw_dtype, lddw, beta, stream);
+}
+
+}  // namespace velora
