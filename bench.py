@@ -341,18 +341,25 @@ def kernel_table(vl, torch, L, N, ws, pk):
     by = {l["name"]: l for l in L}
     out = []
 
-    def timed(fn_list, reps=5):
+    def timed(fn_list, reps=7):
+        """Median device time of one call (ms): every call is bracketed by its own pair of CUDA events."""
         for f in fn_list:
             f()
         torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
+        # Keep the GPU busy for ~2 ms first, so that every call below is already queued when its turn
+        # comes: the event pairs then time device work only, not the host's submission latency.
+        torch.cuda._sleep(4_000_000)
+        pairs = []
         for _ in range(reps):
             for f in fn_list:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
                 f()
-        b.record()
+                b.record()
+                pairs.append((a, b))
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / (reps * len(fn_list))
+        times = sorted(a.elapsed_time(b) for a, b in pairs)
+        return times[len(times) // 2]
 
     def hbm(name, shape, ms, nbytes):
         gbs = nbytes / (ms * 1e-3) / 1e9
@@ -408,14 +415,63 @@ def kernel_table(vl, torch, L, N, ws, pk):
     return out
 
 
+def run_profile(args):
+    """A few launches of one entry point on one config-5 layer: the small, self-ending case for ncu."""
+    import torch
+
+    import paper_2405_17991_b200 as vl
+    import velora_inputs as vi
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = vi.CONFIGS[CONFIG_INDEX]
+    name = {"compress": "down", "reconstruct": "down", "init_v": "down", "weight_grad": "up",
+            "forward": "q", "input_grad": "q", "weight_grad_explicit": "q"}[args.profile]
+    li = [l.name for l in cfg.layers].index(name)
+    layer = cfg.layers[li]
+    N = cfg.N
+    X = vi.make_X(cfg, li).torch(dev)
+    v = vl.velora_init_v(X, DSUB)
+    Z = vl.velora_compress(X, v)
+    ws = vl.velora_workspace_alloc(
+        max(vl.velora_workspace_bytes(op, N, layer.D, layer.O, DSUB)
+            for op in (vl.OP_INIT_V, vl.OP_LINEAR_BACKWARD_FACTORED, vl.OP_WEIGHT_GRAD_EXPLICIT)), dev)
+    if args.profile in ("compress", "reconstruct", "init_v"):
+        Xhat = torch.empty_like(X)
+        fn = {"compress": lambda: vl.velora_compress(X, v, Z=Z),
+              "reconstruct": lambda: vl.velora_reconstruct(Z, v, layer.D, Xhat=Xhat),
+              "init_v": lambda: vl.velora_init_v(X, DSUB, v=v, ws=ws)}[args.profile]
+    else:
+        W = vi.make_W(cfg, li).torch(dev)
+        dY = vi.make_dY(cfg, li).torch(dev)
+        Y = torch.empty((N, layer.O), dtype=torch.bfloat16, device=dev)
+        dX = torch.empty_like(X)
+        dW = torch.empty_like(W)
+        fn = {"weight_grad": lambda: vl.velora_weight_grad(dY, Z, v, layer.D, dW=dW, ws=ws),
+              "weight_grad_explicit": lambda: vl.velora_weight_grad(dY, Z, v, layer.D, dW=dW, mode=vl.WG_EXPLICIT, ws=ws),
+              "forward": lambda: vl.velora_linear_forward(X, W, v, Y=Y, Z=Z, ws=ws),
+              "input_grad": lambda: vl.velora_linear_backward(dY, W, Z, v, dX=dX, need_dW=False, ws=ws)}[args.profile]
+    for _ in range(4):
+        fn()
+    torch.cuda.synchronize()
+    print(json.dumps({"profile": args.profile, "layer": name, "N": N, "D": layer.D, "O": layer.O,
+                      "status": vl.velora_workspace_status(ws)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile", default=None,
+                    choices=["compress", "reconstruct", "init_v", "weight_grad", "weight_grad_explicit",
+                             "forward", "input_grad"],
+                    help="run four launches of one entry point on one layer (for ncu) and exit")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile:
+        run_profile(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

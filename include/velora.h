@@ -105,6 +105,13 @@ int velora_workspace_init(void* ws, size_t ws_bytes, void* stream);
 int velora_workspace_status(const void* ws, void* stream);
 
 /*
+ * The entry points that take no workspace (velora_compress, and velora_init_v's first pass) record an
+ * expired bounded wait in a word inside the library instead.  velora_device_error synchronises
+ * `stream`, returns VELORA_OK or VELORA_ERR_TIMEOUT for the current device and clears the word.
+ */
+int velora_device_error(void* stream);
+
+/*
  * Initialise the projection vector from a batch (Section 3.2, "Cheap
  * initialisation strategies": the average of the first batch's sub-tokens;
  * Section 3.1: v has unit length):

@@ -34,6 +34,7 @@ SIGNATURES = {
     "velora_linear_step_host": (_int, [_p, _p, _p, _p, _p, _p, _p, _p, _sz, _i64, _i64, _i64, _int, _p, _sz, _p]),
     "velora_workspace_init": (_int, [_p, _sz, _p]),
     "velora_workspace_status": (_int, [_p, _p]),
+    "velora_device_error": (_int, [_p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
     "velora_init_v_static": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
@@ -123,6 +124,11 @@ def velora_workspace_init(ws: torch.Tensor, stream=None) -> None:
 def velora_workspace_status(ws: torch.Tensor, stream=None) -> int:
     """Synchronises the stream; 0 or ERR_TIMEOUT if a kernel's bounded wait expired."""
     return int(lib().velora_workspace_status(ctypes.c_void_p(ws.data_ptr()), _stream(stream)))
+
+
+def velora_device_error(stream=None) -> int:
+    """Synchronises the stream; 0, or ERR_TIMEOUT if a streaming kernel's bounded wait expired (then cleared)."""
+    return int(lib().velora_device_error(_stream(stream)))
 
 
 def _check(status: int, where: str):

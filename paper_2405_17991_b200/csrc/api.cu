@@ -135,6 +135,11 @@ int velora_workspace_init(void* ws, size_t ws_bytes, void* stream)
                                                                                                    : VELORA_ERR_CUDA;
 }
 
+int velora_device_error(void* stream)
+{
+    return read_and_clear_stream_error(static_cast<cudaStream_t>(stream));
+}
+
 int velora_workspace_status(const void* ws, void* stream)
 {
     if (!ws) return VELORA_ERR_WORKSPACE;

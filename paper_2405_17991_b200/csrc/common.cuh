@@ -51,6 +51,13 @@ int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ld
                     int64_t O, int64_t D, int Dsub, void* dW, int dw_dtype, int64_t lddw, int beta,
                     cudaStream_t stream);
 
+// Vector form of "row of scalars times v": out[r, m*Dsub + j] = beta*out + (sum_s S[s][r][m]) * v[j] for bf16 or
+// fp32 S (one split: reconstruct; several: the factored weight gradient).  VELORA_ERR_UNSUPPORTED if the shape
+// needs the element-wise kernels.  (expand_kernels.cu)
+int launch_expand_rows_vec(const void* S, int s_dtype, int splits, int64_t split_stride, int64_t lds, const float* v,
+                           int64_t R, int64_t D, int Dsub, void* out, int out_dtype, int64_t ldo, int beta,
+                           cudaStream_t stream);
+
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)

@@ -23,15 +23,27 @@ int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t 
                    int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream);
 
 // Tensor map of a row-major bf16 matrix: `inner` contiguous elements per row, `outer` rows, row pitch
-// ld_elems; 128-byte swizzle, zero fill outside the matrix.  (gemm_tc.cu)
+// ld_elems; 128-byte swizzle (or none), zero fill outside the matrix.  (gemm_tc.cu)
 int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
-                      int box_inner, int box_outer);
+                      int box_inner, int box_outer, bool swizzle128 = true);
 bool tc_operand_ok(const void* p, int64_t ld_elems);
 
 // Y = X W^T with compress(X, v) computed from the same staged X tiles.
 int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
                              void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
                              int dtype, int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
+
+// TMA-staged streaming kernels (stream_tma.cu): X tiles flow through a shared-memory ring.
+// Return VELORA_ERR_UNSUPPORTED (nothing launched) when the shape does not fit them.
+int launch_compress_tma(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                        void* Z, int z_dtype, int64_t ldz, int* status, cudaStream_t stream);
+int launch_init_v_partials_tma(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                               float* partials, int max_partials, int* num_partials, int* status,
+                               cudaStream_t stream);
+
+// Reads (synchronising `stream`) and clears the device word in which the streaming kernels record an
+// expired wait: VELORA_OK or VELORA_ERR_TIMEOUT.
+int read_and_clear_stream_error(cudaStream_t stream);
 
 // Factored weight gradient: P = dY^T Z on tensor cores (split over tokens), dW = P (x) v.
 size_t weight_grad_tc_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub);

@@ -1,19 +1,22 @@
-// HBM-bound streaming kernels of the VeLoRA path: init_v, compress, reconstruct
-// (arxiv 2405.17991, Section 3.1 Eq. 1 / Eq. 2, Section 3.2 initialisation).
+// HBM-bound streaming kernels of the VeLoRA path: init_v, compress, reconstruct and the expansion
+// of the factored weight gradient (arxiv 2405.17991, Section 3.1 Eq. 1 / Eq. 2, Section 3.2).
 //
-// Vector kernels.  A row of X is a sequence of 16-byte chunks (8 bf16).  A
-// sub-token of length Dsub = 8*L is covered by LPS = min(L, 32) adjacent lanes,
-// each lane owning CH = L / LPS chunks, so a warp instruction reads one
-// contiguous 512-byte span.  Work items (row, m, lane-in-group) are numbered
-// row-major and walked with a grid-wide stride that is a multiple of 32: a
-// thread therefore keeps the same position inside its sub-token for the whole
-// kernel and holds its slice of v in registers.  The walk carries (row, pos)
-// incrementally -- no division in the loop.  When Dsub does not divide D the
-// last sub-token's missing chunks are simply not loaded (zero extension).
+// Vector kernels.  A row of X is a sequence of 16-byte chunks (8 bf16).  A sub-token of length
+// Dsub = 8*L is covered by LPS = min(L, 32) adjacent lanes, each lane owning CH = L / LPS chunks, so
+// a warp instruction touches one contiguous 512-byte span.  Work items (row, m, lane-in-group) are
+// numbered row-major and walked with a grid-wide stride that is a multiple of 32: a thread keeps the
+// same position inside its sub-token for the whole kernel and holds its slice of v in registers.  The
+// walk carries (row, pos) incrementally in 32-bit integers -- no division, no 64-bit multiply in the
+// loop (the host cuts very large inputs into launches whose offsets fit 31 bits).  Loads are software
+// pipelined: the next batch of 16-byte loads is issued before the current batch is reduced, so a
+// thread always has loads in flight.  When Dsub does not divide D the last sub-token's missing chunks
+// are not loaded (zero extension); that case uses the RAGGED instances, the common case carries no
+// bounds checks on columns.
 //
-// Element kernels cover everything else (fp32 data, Dsub not a multiple of 8,
-// unaligned rows) with the same arithmetic, one element per lane.
+// Element kernels cover everything else (fp32 data, Dsub not a multiple of 8, unaligned rows) with
+// the same arithmetic, one element per lane.
 #include "common.cuh"
+#include "gemm_tc.cuh"
 
 namespace velora {
 
@@ -23,8 +26,7 @@ constexpr unsigned kFull = 0xffffffffu;
 
 // Walks items tid, tid + S, tid + 2S, ... as (row, pos), pos in [0, items_per_row).
 struct ItemWalk {
-    int64_t row;
-    int pos;
+    int row, pos;
     int row_step, pos_step, ipr;
     __device__ __forceinline__ void init(int items_per_row)
     {
@@ -32,7 +34,7 @@ struct ItemWalk {
         const int S = gridDim.x * blockDim.x;
         ipr = items_per_row;
         row = tid / ipr;
-        pos = tid - static_cast<int>(row) * ipr;
+        pos = tid - row * ipr;
         row_step = S / ipr;
         pos_step = S - row_step * ipr;
     }
@@ -53,7 +55,7 @@ __device__ __forceinline__ void unpack8(const uint4& c, float (&x)[8])
 }
 
 // Loads chunk `chunk` of a row, zeroing whatever lies at or beyond column D.
-__device__ __forceinline__ uint4 load_chunk(const uint4* row_ptr, int chunk, int D)
+__device__ __forceinline__ uint4 load_chunk_ragged(const uint4* row_ptr, int chunk, int D)
 {
     const int col = chunk * 8;
     uint4 c = make_uint4(0u, 0u, 0u, 0u);
@@ -73,15 +75,29 @@ __device__ __forceinline__ uint4 load_chunk(const uint4* row_ptr, int chunk, int
     return c;
 }
 
+template <bool RAGGED>
+__device__ __forceinline__ uint4 load_chunk(const uint4* row_ptr, int chunk, int D)
+{
+    if (RAGGED) return load_chunk_ragged(row_ptr, chunk, D);
+    return __ldg(row_ptr + chunk);
+}
+
 template <typename ZT> __device__ __forceinline__ void store_z(ZT* p, float z);
 template <> __device__ __forceinline__ void store_z<float>(float* p, float z) { *p = z; }
 template <> __device__ __forceinline__ void store_z<__nv_bfloat16>(__nv_bfloat16* p, float z) { *p = __float2bfloat16_rn(z); }
 
+template <typename ZT> __device__ __forceinline__ float load_z(const ZT* p);
+template <> __device__ __forceinline__ float load_z<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float load_z<__nv_bfloat16>(const __nv_bfloat16* p)
+{
+    return __bfloat162float(*p);
+}
+
 // ------------------------------------------------------------------ compress (vector)
-template <int LPS, int CH, int U, typename ZT>
+template <int LPS, int CH, int U, bool RAGGED, typename ZT>
 __global__ void __launch_bounds__(kStreamThreads)
-compress_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldx_chunks, int M,
-                    const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz)
+compress_vec_kernel(const uint4* __restrict__ X, int N, int D, int ldx_chunks, int M,
+                    const float* __restrict__ v, ZT* __restrict__ Z, int ldz)
 {
     constexpr int L = LPS * CH;                  // chunks per sub-token
     const int q = threadIdx.x & (LPS - 1);       // fixed position inside the sub-token
@@ -93,112 +109,54 @@ compress_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldx_c
 
     ItemWalk w;
     w.init(M * LPS);
-    while (__any_sync(kFull, w.row < N)) {
-        uint4 data[U][CH];
-        int64_t rows[U];
-        int ms[U];
+    // One batch = U items per thread; zoff is the item's offset in Z, or -1 past the end.
+    auto fetch = [&](uint4 (&d)[U][CH], int (&zoff)[U]) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            rows[u] = w.row;
-            ms[u] = w.pos / LPS;                 // LPS is a power of two
             const bool valid = w.row < N;
-            const uint4* rp = X + w.row * ldx_chunks;
+            const int m = w.pos / LPS;           // LPS is a power of two
+            zoff[u] = valid ? w.row * ldz + m : -1;
+            const uint4* rp = X + (valid ? w.row * ldx_chunks : 0);
 #pragma unroll
             for (int i = 0; i < CH; ++i)
-                data[u][i] = valid ? load_chunk(rp, ms[u] * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
+                d[u][i] = valid ? load_chunk<RAGGED>(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
             w.advance();
         }
+    };
+    uint4 cur[U][CH];
+    int czoff[U];
+    fetch(cur, czoff);
+    while (__any_sync(kFull, czoff[0] >= 0)) {
+        uint4 nxt[U][CH];
+        int nzoff[U];
+        fetch(nxt, nzoff);                       // next batch in flight while this one is reduced
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             float acc = 0.f;
 #pragma unroll
             for (int i = 0; i < CH; ++i) {
                 float x[8];
-                unpack8(data[u][i], x);
+                unpack8(cur[u][i], x);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc = fmaf(x[e], vr[i][e], acc);
             }
 #pragma unroll
             for (int off = LPS / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(kFull, acc, off);
-            if (q == 0 && rows[u] < N) store_z<ZT>(Z + rows[u] * ldz + ms[u], acc);
-        }
-    }
-}
-
-// ------------------------------------------------------------------ reconstruct (vector, bf16 out)
-template <typename ZT> __device__ __forceinline__ float load_z(const ZT* p);
-template <> __device__ __forceinline__ float load_z<float>(const float* p) { return __ldg(p); }
-template <> __device__ __forceinline__ float load_z<__nv_bfloat16>(const __nv_bfloat16* p)
-{
-    return __bfloat162float(*p);
-}
-
-__device__ __forceinline__ void store_chunk_bf16(uint4* row_ptr, __nv_bfloat16* row_elems, int chunk, int D,
-                                                 const float (&y)[8])
-{
-    const int col = chunk * 8;
-    if (col + 8 <= D) {
-        uint4 o;
-        o.x = pack_bf16x2(y[0], y[1]);
-        o.y = pack_bf16x2(y[2], y[3]);
-        o.z = pack_bf16x2(y[4], y[5]);
-        o.w = pack_bf16x2(y[6], y[7]);
-        __stcs(row_ptr + chunk, o);
-    } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e)
-            if (col + e < D) row_elems[col + e] = __float2bfloat16_rn(y[e]);
-    }
-}
-
-template <int LPS, int CH, int U, typename ZT>
-__global__ void __launch_bounds__(kStreamThreads)
-reconstruct_vec_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D, int M,
-                       const float* __restrict__ v, uint4* __restrict__ Xhat, int64_t ldx_chunks)
-{
-    constexpr int L = LPS * CH;
-    const int q = threadIdx.x & (LPS - 1);
-    float vr[CH][8];
-#pragma unroll
-    for (int i = 0; i < CH; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
-
-    ItemWalk w;
-    w.init(M * LPS);
-    while (w.row < N) {
-        float z[U];
-        int64_t rows[U];
-        int ms[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            rows[u] = w.row;
-            ms[u] = w.pos / LPS;
-            z[u] = (w.row < N) ? load_z<ZT>(Z + w.row * ldz + ms[u]) : 0.f;
-            w.advance();
+            if (q == 0 && czoff[u] >= 0) store_z<ZT>(Z + czoff[u], acc);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (rows[u] < N) {
-                uint4* rp = Xhat + rows[u] * ldx_chunks;
-                __nv_bfloat16* re = reinterpret_cast<__nv_bfloat16*>(rp);
+            czoff[u] = nzoff[u];
 #pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    float y[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = z[u] * vr[i][e];
-                    const int chunk = ms[u] * L + q + LPS * i;
-                    if (chunk * 8 < D) store_chunk_bf16(rp, re, chunk, D, y);
-                }
-            }
+            for (int i = 0; i < CH; ++i) cur[u][i] = nxt[u][i];
         }
     }
 }
 
 // ------------------------------------------------------------------ init_v (vector): per-CTA partial sums
-template <int LPS, int CH, int U>
+template <int LPS, int CH, int U, bool RAGGED>
 __global__ void __launch_bounds__(kStreamThreads)
-init_v_partial_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldx_chunks, int M,
+init_v_partial_vec_kernel(const uint4* __restrict__ X, int N, int D, int ldx_chunks, int M,
                           float* __restrict__ partials /* [gridDim.x][8*L] */)
 {
     constexpr int L = LPS * CH;
@@ -212,26 +170,34 @@ init_v_partial_vec_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t
 
     ItemWalk w;
     w.init(M * LPS);
-    while (w.row < N) {
-        uint4 data[U][CH];
+    auto fetch = [&](uint4 (&d)[U][CH]) -> bool {
+        const bool any = w.row < N;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const bool valid = w.row < N;
-            const uint4* rp = X + w.row * ldx_chunks;
+            const uint4* rp = X + (valid ? w.row * ldx_chunks : 0);
             const int m = w.pos / LPS;
 #pragma unroll
             for (int i = 0; i < CH; ++i)
-                data[u][i] = valid ? load_chunk(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
+                d[u][i] = valid ? load_chunk<RAGGED>(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
             w.advance();
         }
+        return any;
+    };
+    uint4 cur[U][CH];
+    bool more = fetch(cur);
+    while (more) {
+        uint4 nxt[U][CH];
+        more = fetch(nxt);
 #pragma unroll
         for (int u = 0; u < U; ++u)
 #pragma unroll
             for (int i = 0; i < CH; ++i) {
                 float x[8];
-                unpack8(data[u][i], x);
+                unpack8(cur[u][i], x);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[i][e] += x[e];
+                cur[u][i] = nxt[u][i];
             }
     }
 
@@ -355,7 +321,8 @@ reconstruct_elem_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D,
     }
 }
 
-// Expansion of the factored weight gradient (Section 3.2's rank-1 form, per sub-token):
+// ------------------------------------------------------------------ expansion of the factored weight gradient
+// (Section 3.2's rank-1 form, per sub-token):
 //   dW[o, m*Dsub + j] = beta*dW[o, m*Dsub + j] + (sum_s P[s][o][m]) * v[j]
 // P holds `splits` partial products dY^T Z over disjoint token ranges, summed here in a fixed order.
 template <typename WT>
@@ -376,99 +343,6 @@ expand_p_elem_kernel(const float* __restrict__ P, int splits, int64_t split_stri
         float r = p * __ldg(v + j);
         if (beta) r += Elem<WT>::load(dW + o * lddw + d);
         Elem<WT>::store(dW + o * lddw + d, r);
-    }
-}
-
-template <typename WT> struct Chunk8;
-template <> struct Chunk8<__nv_bfloat16> {
-    static __device__ __forceinline__ void store(__nv_bfloat16* row, int col, float (&y)[8], int beta)
-    {
-        uint4* p = reinterpret_cast<uint4*>(row + col);
-        if (beta) {
-            const uint4 old = *p;
-            y[0] += bf16_lo(old.x); y[1] += bf16_hi(old.x);
-            y[2] += bf16_lo(old.y); y[3] += bf16_hi(old.y);
-            y[4] += bf16_lo(old.z); y[5] += bf16_hi(old.z);
-            y[6] += bf16_lo(old.w); y[7] += bf16_hi(old.w);
-        }
-        uint4 o;
-        o.x = pack_bf16x2(y[0], y[1]);
-        o.y = pack_bf16x2(y[2], y[3]);
-        o.z = pack_bf16x2(y[4], y[5]);
-        o.w = pack_bf16x2(y[6], y[7]);
-        __stcs(p, o);
-    }
-};
-template <> struct Chunk8<float> {
-    static __device__ __forceinline__ void store(float* row, int col, float (&y)[8], int beta)
-    {
-        float4* p = reinterpret_cast<float4*>(row + col);
-        if (beta) {
-            const float4 a = p[0], b = p[1];
-            y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
-            y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
-        }
-        __stcs(p, make_float4(y[0], y[1], y[2], y[3]));
-        __stcs(p + 1, make_float4(y[4], y[5], y[6], y[7]));
-    }
-};
-
-// Vector form: same item walk as reconstruct, rows are output rows o.
-template <int LPS, int CH, int U, typename WT>
-__global__ void __launch_bounds__(kStreamThreads)
-expand_p_vec_kernel(const float* __restrict__ P, int splits, int64_t split_stride, int64_t ldp,
-                    const float* __restrict__ v, int64_t O, int D, int M,
-                    WT* __restrict__ dW, int64_t lddw, int beta)
-{
-    constexpr int L = LPS * CH;
-    const int q = threadIdx.x & (LPS - 1);
-    float vr[CH][8];
-#pragma unroll
-    for (int i = 0; i < CH; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
-
-    ItemWalk w;
-    w.init(M * LPS);
-    while (w.row < O) {
-        float p[U];
-        int64_t rows[U];
-        int ms[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            rows[u] = w.row;
-            ms[u] = w.pos / LPS;
-            p[u] = 0.f;
-            if (w.row < O) {
-                const float* pp = P + w.row * ldp + ms[u];
-                for (int s = 0; s < splits; ++s) p[u] += __ldg(pp + s * split_stride);
-            }
-            w.advance();
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (rows[u] < O) {
-                WT* row = dW + rows[u] * lddw;
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int col = (ms[u] * L + q + LPS * i) * 8;
-                    float y[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = p[u] * vr[i][e];
-                    if (col + 8 <= D) {
-                        Chunk8<WT>::store(row, col, y, beta);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            if (col + e < D) {
-                                float r = y[e];
-                                if (beta) r += Elem<WT>::load(row + col + e);
-                                Elem<WT>::store(row + col + e, r);
-                            }
-                    }
-                }
-            }
-        }
     }
 }
 
@@ -515,10 +389,15 @@ int check_launch()
     return after_launch();
 }
 
-// Largest number of rows one vector launch may take so that item counts stay below 2^30.
-int64_t max_rows_per_launch(int items_per_row)
+// Largest number of rows one vector launch may take so that item counts and the element offsets
+// row*ld_a, row*ld_b stay within 31 bits.
+int64_t max_rows_per_launch(int items_per_row, int64_t ld_a, int64_t ld_b)
 {
-    return (static_cast<int64_t>(1) << 30) / items_per_row;
+    int64_t r = (static_cast<int64_t>(1) << 30) / items_per_row;
+    const int64_t lim = (static_cast<int64_t>(1) << 31) - 1;
+    if (ld_a > 0 && lim / ld_a < r) r = lim / ld_a;
+    if (ld_b > 0 && lim / ld_b < r) r = lim / ld_b;
+    return r < 1 ? 1 : r;
 }
 
 #define VELORA_DISPATCH_VEC(SHAPE, KERNEL_CALL)                                              \
@@ -549,20 +428,31 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
     const int M = static_cast<int>(ceil_div64(D, Dsub));
     const VecShape vs = vec_shape(Dsub);
+    const bool ragged = (D % Dsub) != 0;
     int num_partials = 0;
 
-    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx) &&
-        N <= max_rows_per_launch(M * vs.lps)) {
+    int tma_rc = VELORA_ERR_UNSUPPORTED;
+    if (x_dtype == VELORA_BF16 && D >= 256)
+        tma_rc = launch_init_v_partials_tma(X, N, D, ldx, Dsub, partials, kInitVMaxCtas, &num_partials, nullptr, stream);
+    if (tma_rc != VELORA_ERR_UNSUPPORTED) {
+        if (tma_rc != VELORA_OK) return tma_rc;
+    } else if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx) &&
+        N <= max_rows_per_launch(M * vs.lps, ldx / 8, 0)) {
         const int64_t items = N * M * vs.lps;
         int grid = 0;
-        int rc = stream_grid(items, vs.u, &grid);
+        int rc = stream_grid(items, 2 * vs.u, &grid);
         if (rc != VELORA_OK) return rc;
         if (grid > kInitVMaxCtas) grid = kInitVMaxCtas;
         num_partials = grid;
         const size_t smem = static_cast<size_t>(kStreamThreads) * 8 * vs.ch * sizeof(float);
+        const int n = static_cast<int>(N), d = static_cast<int>(D), ldc = static_cast<int>(ldx / 8);
 #define CALL_INIT(LPS, CH, U)                                                                             \
-        init_v_partial_vec_kernel<LPS, CH, U><<<grid, kStreamThreads, smem, stream>>>(                    \
-            static_cast<const uint4*>(X), N, static_cast<int>(D), ldx / 8, M, partials)
+        if (ragged)                                                                                       \
+            init_v_partial_vec_kernel<LPS, CH, U, true><<<grid, kStreamThreads, smem, stream>>>(          \
+                static_cast<const uint4*>(X), n, d, ldc, M, partials);                                    \
+        else                                                                                              \
+            init_v_partial_vec_kernel<LPS, CH, U, false><<<grid, kStreamThreads, smem, stream>>>(         \
+                static_cast<const uint4*>(X), n, d, ldc, M, partials)
         VELORA_DISPATCH_VEC(vs, CALL_INIT)
 #undef CALL_INIT
     } else {
@@ -599,23 +489,34 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
 {
     const int M = static_cast<int>(ceil_div64(D, Dsub));
     const VecShape vs = vec_shape(Dsub);
+    const bool ragged = (D % Dsub) != 0;
+    if (x_dtype == VELORA_BF16 && D >= 256) {            // TMA-staged kernel: large rows, Dsub in {8..256}
+        const int rc = launch_compress_tma(X, N, D, ldx, Dsub, v, Z, z_dtype, ldz, nullptr, stream);
+        if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    }
     if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx)) {
-        const int64_t step = max_rows_per_launch(M * vs.lps);
+        const int64_t step = max_rows_per_launch(M * vs.lps, ldx / 8, ldz);
+        const int d = static_cast<int>(D), ldc = static_cast<int>(ldx / 8), ldzi = static_cast<int>(ldz);
         for (int64_t r0 = 0; r0 < N; r0 += step) {
-            const int64_t n = (N - r0 < step) ? N - r0 : step;
+            const int n = static_cast<int>((N - r0 < step) ? N - r0 : step);
             int grid = 0;
-            int rc = stream_grid(n * M * vs.lps, vs.u, &grid);
+            int rc = stream_grid(static_cast<int64_t>(n) * M * vs.lps, 2 * vs.u, &grid);
             if (rc != VELORA_OK) return rc;
             const uint4* xp = static_cast<const uint4*>(X) + r0 * (ldx / 8);
+#define CALL_COMPRESS_T(LPS, CH, U, RAG, ZT)                                                              \
+            compress_vec_kernel<LPS, CH, U, RAG, ZT><<<grid, kStreamThreads, 0, stream>>>(                \
+                xp, n, d, ldc, M, v, static_cast<ZT*>(Z) + r0 * ldz, ldzi)
 #define CALL_COMPRESS(LPS, CH, U)                                                                         \
-            if (z_dtype == VELORA_F32)                                                                    \
-                compress_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(              \
-                    xp, n, static_cast<int>(D), ldx / 8, M, v, static_cast<float*>(Z) + r0 * ldz, ldz);   \
-            else                                                                                          \
-                compress_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(      \
-                    xp, n, static_cast<int>(D), ldx / 8, M, v, static_cast<__nv_bfloat16*>(Z) + r0 * ldz, ldz)
+            if (z_dtype == VELORA_F32) {                                                                  \
+                if (ragged) CALL_COMPRESS_T(LPS, CH, U, true, float);                                     \
+                else CALL_COMPRESS_T(LPS, CH, U, false, float);                                           \
+            } else {                                                                                      \
+                if (ragged) CALL_COMPRESS_T(LPS, CH, U, true, __nv_bfloat16);                             \
+                else CALL_COMPRESS_T(LPS, CH, U, false, __nv_bfloat16);                                   \
+            }
             VELORA_DISPATCH_VEC(vs, CALL_COMPRESS)
 #undef CALL_COMPRESS
+#undef CALL_COMPRESS_T
             if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
         }
         return VELORA_OK;
@@ -637,28 +538,9 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
 int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
                        const float* v, void* Xhat, int x_dtype, int64_t ldxhat, cudaStream_t stream)
 {
-    const int M = static_cast<int>(ceil_div64(D, Dsub));
-    const VecShape vs = vec_shape(Dsub);
-    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(Xhat, ldxhat)) {
-        const int64_t step = max_rows_per_launch(M * vs.lps);
-        for (int64_t r0 = 0; r0 < N; r0 += step) {
-            const int64_t n = (N - r0 < step) ? N - r0 : step;
-            int grid = 0;
-            int rc = stream_grid(n * M * vs.lps, vs.u, &grid);
-            if (rc != VELORA_OK) return rc;
-            uint4* xp = static_cast<uint4*>(Xhat) + r0 * (ldxhat / 8);
-#define CALL_RECON(LPS, CH, U)                                                                            \
-            if (z_dtype == VELORA_F32)                                                                    \
-                reconstruct_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(           \
-                    static_cast<const float*>(Z) + r0 * ldz, ldz, n, static_cast<int>(D), M, v, xp, ldxhat / 8); \
-            else                                                                                          \
-                reconstruct_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(   \
-                    static_cast<const __nv_bfloat16*>(Z) + r0 * ldz, ldz, n, static_cast<int>(D), M, v, xp, ldxhat / 8)
-            VELORA_DISPATCH_VEC(vs, CALL_RECON)
-#undef CALL_RECON
-            if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
-        }
-        return VELORA_OK;
+    if (x_dtype == VELORA_BF16) {                        // Xhat = Z (x) v is the one-split, beta = 0 expansion
+        const int rc = launch_expand_rows_vec(Z, z_dtype, 1, 0, ldz, v, N, D, Dsub, Xhat, x_dtype, ldxhat, 0, stream);
+        if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     }
     int grid = 0;
     int rc = stream_grid(N * D, 4, &grid);
@@ -678,26 +560,10 @@ int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ld
                     int64_t O, int64_t D, int Dsub, void* dW, int dw_dtype, int64_t lddw, int beta,
                     cudaStream_t stream)
 {
-    const int M = static_cast<int>(ceil_div64(D, Dsub));
-    const VecShape vs = vec_shape(Dsub);
-    const bool rows16 = aligned16(dW) && (lddw * static_cast<int64_t>(dtype_size(dw_dtype))) % 16 == 0;
-    if (vs.ok && rows16 && O <= max_rows_per_launch(M * vs.lps)) {
-        int grid = 0;
-        int rc = stream_grid(O * M * vs.lps, vs.u, &grid);
-        if (rc != VELORA_OK) return rc;
-#define CALL_EXPAND(LPS, CH, U)                                                                            \
-        if (dw_dtype == VELORA_BF16)                                                                       \
-            expand_p_vec_kernel<LPS, CH, U, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(           \
-                P, splits, split_stride, ldp, v, O, static_cast<int>(D), M, static_cast<__nv_bfloat16*>(dW), lddw, beta); \
-        else                                                                                               \
-            expand_p_vec_kernel<LPS, CH, U, float><<<grid, kStreamThreads, 0, stream>>>(                   \
-                P, splits, split_stride, ldp, v, O, static_cast<int>(D), M, static_cast<float*>(dW), lddw, beta)
-        VELORA_DISPATCH_VEC(vs, CALL_EXPAND)
-#undef CALL_EXPAND
-        return check_launch();
-    }
+    int rc = launch_expand_rows_vec(P, VELORA_F32, splits, split_stride, ldp, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     int grid = 0;
-    int rc = stream_grid(O * D, 4, &grid);
+    rc = stream_grid(O * D, 4, &grid);
     if (rc != VELORA_OK) return rc;
     if (dw_dtype == VELORA_BF16)
         expand_p_elem_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(
@@ -709,7 +575,6 @@ int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ld
 }
 
 }  // namespace velora
-
 // ------------------------------------------------------------------ velora_init_v without a workspace
 // Scratch for velora_init_v_static: the status header plus one row of partial sums per CTA, for
 // sub-tokens of up to VELORA_INIT_V_STATIC_MAX_DSUB elements.  It is part of the loaded module, so
