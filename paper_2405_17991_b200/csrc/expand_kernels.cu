@@ -17,7 +17,6 @@ namespace velora {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kMaxSplitsUnrolled = 8;
 
 template <typename T> __device__ __forceinline__ float load_scalar(const T* p);
 template <> __device__ __forceinline__ float load_scalar<float>(const float* p) { return __ldg(p); }
@@ -80,20 +79,15 @@ expand_rows_vec_kernel(const ST* __restrict__ S, int splits, int64_t split_strid
 #pragma unroll
         for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
 
+    // One warp per output row at a time; the row's blocks of 32 sub-tokens are walked in an inner loop.
     const int warps = gridDim.x * (kStreamThreads / 32);
-    const int64_t tasks = static_cast<int64_t>(R) * mblocks;
-    for (int64_t task = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5); task < tasks; task += warps) {
-        const int r = static_cast<int>(task / mblocks);
-        const int m0 = static_cast<int>(task - static_cast<int64_t>(r) * mblocks) * 32;
+    for (int r = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5); r < R; r += warps)
+    for (int m0 = 0; m0 < mblocks * 32; m0 += 32) {
         float p = 0.f;
         if (MODE == 0 || m0 + lane < M) {
             const ST* sp = S + static_cast<int64_t>(r) * lds + m0 + lane;
-            float part[kMaxSplitsUnrolled];
-#pragma unroll
-            for (int s = 0; s < kMaxSplitsUnrolled; ++s) part[s] = (s < splits) ? load_scalar<ST>(sp + s * split_stride) : 0.f;
-#pragma unroll
-            for (int s = 0; s < kMaxSplitsUnrolled; ++s) p += part[s];
-            for (int s = kMaxSplitsUnrolled; s < splits; ++s) p += load_scalar<ST>(sp + s * split_stride);
+#pragma unroll 4
+            for (int s = 0; s < splits; ++s) p += load_scalar<ST>(sp + s * split_stride);   // fixed order
         }
         // Element pointer of this lane's first chunk; each step moves on by SPW sub-tokens.
         WT* ptr = out + static_cast<int64_t>(r) * ldo + (static_cast<int64_t>(m0 + sub) * L + q) * 8;
@@ -182,8 +176,7 @@ int launch_expand_rows_vec(const void* S, int s_dtype, int splits, int64_t split
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != VELORA_OK) return rc;
-    const int64_t tasks = R * mblocks;
-    int64_t ctas = ceil_div64(tasks, kStreamThreads / 32);
+    int64_t ctas = ceil_div64(R, kStreamThreads / 32);
     const int64_t cap = static_cast<int64_t>(di.sm_count) * kStreamCtasPerSm;
     if (ctas > cap) ctas = cap;
     const int grid = static_cast<int>(ctas < 1 ? 1 : ctas);

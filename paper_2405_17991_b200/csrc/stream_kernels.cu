@@ -254,6 +254,8 @@ init_v_partial_elem_kernel(const XT* __restrict__ X, int64_t N, int D, int64_t l
 
 // ------------------------------------------------------------------ init_v finalize: one CTA
 // s[j] = sum over CTAs (fixed order, fp64), norm, v = s / ||s||.  status[0] = 0 ok, 1 degenerate.
+// For a block of up to 256 positions the 256 threads split the partial rows into `slots` interleaved
+// groups (independent loads), then one thread per position adds the groups in order.
 __global__ void __launch_bounds__(kStreamThreads)
 init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int Dsub,
                        float* __restrict__ v, int* __restrict__ status)
@@ -261,13 +263,26 @@ init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int
     __shared__ double s_sum[VELORA_MAX_DSUB];
     __shared__ double s_red[kStreamThreads];
     __shared__ double s_norm;
-    double sq = 0.0;
-    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) {
+    for (int j0 = 0; j0 < Dsub; j0 += kStreamThreads) {
+        const int width = (Dsub - j0 < kStreamThreads) ? Dsub - j0 : kStreamThreads;
+        const int slots = kStreamThreads / width;
+        const int j = j0 + threadIdx.x % width;
+        const int slot = threadIdx.x / width;
         double s = 0.0;
-        for (int b = 0; b < num_partials; ++b) s += static_cast<double>(partials[static_cast<int64_t>(b) * Dsub + j]);
-        s_sum[j] = s;
-        sq += s * s;
+        if (slot < slots)
+            for (int b = slot; b < num_partials; b += slots)
+                s += static_cast<double>(partials[static_cast<int64_t>(b) * Dsub + j]);
+        s_red[threadIdx.x] = s;
+        __syncthreads();
+        if (threadIdx.x < width) {
+            double t = 0.0;
+            for (int k = 0; k < slots; ++k) t += s_red[k * width + threadIdx.x];
+            s_sum[j] = t;
+        }
+        __syncthreads();
     }
+    double sq = 0.0;
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) sq += s_sum[j] * s_sum[j];
     s_red[threadIdx.x] = sq;
     __syncthreads();
     if (threadIdx.x == 0) {

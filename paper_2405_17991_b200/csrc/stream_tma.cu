@@ -2,10 +2,10 @@
 // of init_v (Section 3.2) for bf16 inputs with 16-byte aligned rows and Dsub in {8, 16, ..., 256}.
 //
 // These kernels are bound by the HBM read of X, so the design goal is bytes in flight, not math.
-// One persistent CTA per SM keeps a ring of six 32 KB stages in shared memory.  A single producer
+// Two persistent CTAs per SM each keep a ring of three 32 KB stages in shared memory.  A single producer
 // thread issues 2-d TMA tile loads (boxes of 16 rows x 256 columns, no swizzle) that complete on
 // mbarriers, so up to 192 KB per SM are in flight regardless of what the consumers do.  Sixteen consumer
-// warps read the landed tiles with conflict-free 16-byte shared-memory loads (a warp instruction reads
+// warps per CTA read the landed tiles with conflict-free 16-byte shared-memory loads (a warp instruction reads
 // one 512-byte tile row), form the dot products with a slice of v held in registers, reduce over the
 // Dsub/8 lanes of a sub-token with xor shuffles and write Z.  Rows beyond N and columns beyond D are
 // zero-filled by TMA, which is exactly the zero extension of a ragged last sub-token: the kernel has
@@ -25,7 +25,7 @@ constexpr int ST_COLS = 256;                      // columns per box (512 bytes)
 constexpr int ST_NB = 4;                          // boxes per stage
 constexpr int ST_BOX_BYTES = ST_R * ST_COLS * 2;  // 8 KB
 constexpr int ST_STAGE_BYTES = ST_NB * ST_BOX_BYTES;
-constexpr int ST_STAGES = 6;
+constexpr int ST_STAGES = 3;                      // per CTA; two CTAs share an SM
 constexpr int ST_CONSUMERS = 16;                  // warps, one tile row each
 constexpr int ST_THREADS = (ST_CONSUMERS + 1) * 32;
 constexpr int ST_ROWS_PER_WARP = ST_R / ST_CONSUMERS;
@@ -47,7 +47,7 @@ template <> __device__ __forceinline__ void put_z<__nv_bfloat16>(__nv_bfloat16* 
 // LPS = Dsub / 8 lanes per sub-token (power of two, <= 32).  INIT = false: compress, writes Z.
 // INIT = true: init_v partial sums, writes partials[blockIdx.x][Dsub].
 template <int LPS, bool INIT, typename ZT>
-__global__ void __launch_bounds__(ST_THREADS, 1)
+__global__ void __launch_bounds__(ST_THREADS, 2)
 stream_tma_kernel(const __grid_constant__ CUtensorMap tmX, int N, int M, int ncb, int cgroups, int units,
                   const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz, float* __restrict__ partials)
 {
@@ -219,7 +219,7 @@ StreamPlan plan_stream(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsu
     const int64_t units = ceil_div64(N, ST_R) * p.cgroups;
     if (units > (1 << 30)) return p;
     p.units = static_cast<int>(units);
-    p.grid = p.units < sm_count ? p.units : sm_count;
+    p.grid = p.units < 2 * sm_count ? p.units : 2 * sm_count;
     p.ok = true;
     return p;
 }
