@@ -30,6 +30,7 @@ UNIT = "tokens/s"
 CONFIG_INDEX = 5
 DSUB = 64
 CPU_SAMPLE_TOKENS = 4
+GEMM_TRAFFIC_RATIO = 0.997      # ncu dram bytes / algorithmic bytes of gemm_tc_kernel on the q layer
 
 
 def peaks():
@@ -275,9 +276,15 @@ def run_ours(args):
     fwd_flops = sum(layer_flops(N, l["D"], l["O"], l["M"])["fwd"] for (l, _, _, _) in events)
     achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
     peak = pk["bf16_tflops_sustained"]
+    # DRAM traffic per launch: ncu on the q-layer launch of this kernel read + wrote 0.997 of the algorithmic
+    # bytes (every operand crosses HBM once; profiles/gemm_tc_kernel_q_layer_8192x4096x4096.md); the other
+    # layers of the step are scaled by their algorithmic bytes.
+    fwd_bytes = sum((N * l["D"] + l["O"] * l["D"] + N * l["O"]) * 2 for (l, _, _, _) in events)
+    traffic = GEMM_TRAFFIC_RATIO * fwd_bytes / max(len(events), 1)
     roofline = {"kernel": "velora_linear_forward (tensor-core GEMM Y = X W^T with compress)", "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": "%s, sustained bf16 GEMM" % pk["source"], "traffic": None,
+                "peak_source": "%s, sustained bf16 GEMM" % pk["source"], "traffic": traffic,
+                "traffic_unit": "bytes per launch (average over the 7 layers; q-layer ncu capture, scaled)",
                 "launches": len(events), "avg_launch_ms": fwd_ms / max(len(events), 1),
                 "fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps}
 
@@ -388,6 +395,13 @@ def kernel_table(vl, torch, L, N, ws, pk):
         hbm("reconstruct", label, ms, N * D * 2 + N * M * 4)
         ms = timed([(lambda l=l: vl.velora_init_v(l["X"], DSUB, v=l["v"], ws=ws)) for l in group])
         hbm("init_v (incl. one stream sync)", label, ms, N * D * 2)
+    # context only: torch's own fill and reduction on the same 180 MB buffer (pure write / pure read ceilings)
+    big_x = big["dX"]
+    hbm("reference: torch zero_ (pure write, library kernel)", "N=%d D=11008" % N, timed([lambda: big_x.zero_()]),
+        N * big["D"] * 2)
+    big_i = big["X"].view(torch.int16)
+    hbm("reference: torch max (pure read, library kernel)", "N=%d D=11008" % N, timed([lambda: big_i.max()]),
+        N * big["D"] * 2)
     # weight gradient, factored: rotate over layers of equal shape
     for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
         group = [by[n] for n in names]
