@@ -24,7 +24,16 @@ constexpr int B_BYTES = BN * BK * 2;              // 32 KB
 constexpr int SLAB_BYTES = 64 * BK * 2;           // one 64-wide MN-major slab: 64 k-rows x 128 bytes
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256;
+constexpr int FUSE_THREADS = GEMM_THREADS + 128;    // + four compress warps
+constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256 + VELORA_MAX_DSUB * 4;
+
+// Arguments of the compress that rides on the forward GEMM's A tiles (Section 3.1, Eq. 1).
+struct FuseArgs {
+    const float* v;
+    void* Z;
+    int64_t ldz;
+    int Dsub, M;
+};
 
 struct TileCoord {
     int m0, n0;
@@ -107,12 +116,19 @@ template <> struct Store32<float> {
     }
 };
 
-template <bool A_MN, bool B_MN, typename CT>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+// FUSE = 0: plain GEMM.  FUSE = 1 / 2 (forward only, A = X K-major): four extra warps read every landed
+// X tile from shared memory and compute Z = compress(X, v) in fp32 / bf16 storage, so X crosses HBM once
+// for both results.  A k-block of 64 columns holds 64/Dsub sub-tokens (or 1/w of one, w = Dsub/64); the
+// CTA working on n-tile j handles the sub-token groups g with g % tiles_n == j, so the work is spread
+// over the CTAs that share a row block.  Thread t of the compress warps owns tile row t; the 128-byte
+// swizzle of the tile makes its 16-byte reads conflict-free.
+template <bool A_MN, bool B_MN, typename CT, int FUSE>
+__global__ void __launch_bounds__(FUSE ? FUSE_THREADS : GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                CT* __restrict__ C, int64_t ldc, int beta, int Mdim, int Ndim, int Kdim,
-               int tiles_m, int tiles_n, int* __restrict__ status)
+               int tiles_m, int tiles_n, int* __restrict__ status, const FuseArgs fz)
 {
+    static_assert(FUSE == 0 || (!A_MN && !B_MN), "compress rides on the K-major forward GEMM only");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;               // swizzled tiles need 1024-byte alignment
@@ -125,6 +141,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tfull = bars + 16 * STAGES, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 40);
+    float* sv = reinterpret_cast<float*>(tail + 256);           // copy of v for the compress warps
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -134,7 +151,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full + 8 * s, 1);
-            mbar_init(empty + 8 * s, 1);
+            mbar_init(empty + 8 * s, FUSE ? 5 : 1);             // MMA commit (+ one arrival per compress warp)
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull + 8 * a, 1);
@@ -149,6 +166,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
+    if (FUSE)
+        for (int j = threadIdx.x; j < fz.Dsub; j += blockDim.x) sv[j] = fz.v[j];
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -226,6 +245,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (failed) *abort_flag = 1;
         }
+    } else if (FUSE && warp >= 6) {
+        // ------------------------------------------------ compress (4 warps, one tile row per thread)
+        const int trow = (warp - 6) * 32 + lane;
+        const int Dsub = fz.Dsub;
+        const int w = Dsub >= BK ? Dsub / BK : 1;              // k-blocks per sub-token
+        const int nsub = Dsub >= BK ? 1 : BK / Dsub;           // sub-tokens per k-block
+        float acc = 0.f;
+        uint32_t it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
+            const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
+            const int tn = tc0.n0 / BN;
+            const int row = tc0.m0 + trow;
+            for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                if (!mbar_wait_warp(full + 8 * s, ph, abort_flag)) { failed = true; break; }
+                const int g = kb / w;
+                if (g % tiles_n == tn) {
+                    const uint32_t rowaddr = sA + s * A_BYTES + trow * 128;
+                    const int j0 = (kb % w) * BK;              // position of this k-block inside the sub-token
+                    if (kb % w == 0) acc = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint4 d;
+                        const uint32_t a = rowaddr + (static_cast<uint32_t>(c ^ (trow & 7)) << 4);
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(d.x), "=r"(d.y), "=r"(d.z), "=r"(d.w) : "r"(a));
+                        const int jv = (j0 + c * 8) % Dsub;    // Dsub and 8 are powers of two here
+                        const float4 va = *reinterpret_cast<const float4*>(sv + jv);
+                        const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
+                        if (nsub > 1 && jv == 0) acc = 0.f;    // a new sub-token starts inside the k-block
+                        acc = fmaf(bf16_lo(d.x), va.x, acc); acc = fmaf(bf16_hi(d.x), va.y, acc);
+                        acc = fmaf(bf16_lo(d.y), va.z, acc); acc = fmaf(bf16_hi(d.y), va.w, acc);
+                        acc = fmaf(bf16_lo(d.z), vb.x, acc); acc = fmaf(bf16_hi(d.z), vb.y, acc);
+                        acc = fmaf(bf16_lo(d.w), vb.z, acc); acc = fmaf(bf16_hi(d.w), vb.w, acc);
+                        // The sub-token ends with this chunk, or the row does (ragged last sub-token: the
+                        // columns beyond D were zero-filled by TMA and no further k-block follows).
+                        if (jv + 8 == Dsub || (kb == kblocks - 1 && c == 7)) {
+                            const int m = (kb * BK + c * 8) / Dsub;
+                            if (row < Mdim && m < fz.M) {
+                                if (FUSE == 1) static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = acc;
+                                else static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + 8 * s);     // this warp is done with the stage
+            }
+        }
+        if (failed) *abort_flag = 1;
     } else {
         // ------------------------------------------------ epilogue (4 warps, one TMEM lane quarter each)
         const int quarter = warp & 3;
@@ -233,7 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x, ++t) {
             const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
             const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
-            if (!mbar_wait(tfull + 8 * acc, aph, abort_flag)) { failed = true; break; }
+            if (!mbar_wait_warp(tfull + 8 * acc, aph, abort_flag)) { failed = true; break; }
             tc_fence_after_sync();
             const int row = tc0.m0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + acc * BN + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -285,14 +354,14 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-template <bool A_MN, bool B_MN, typename CT>
+template <bool A_MN, bool B_MN, typename CT, int FUSE = 0>
 int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t ldc, int beta,
-                  int Mdim, int Ndim, int Kdim, int* status, cudaStream_t stream)
+                  int Mdim, int Ndim, int Kdim, int* status, cudaStream_t stream, const FuseArgs fz = FuseArgs{})
 {
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
-    auto kern = gemm_tc_kernel<A_MN, B_MN, CT>;
+    auto kern = gemm_tc_kernel<A_MN, B_MN, CT, FUSE>;
     if (!configured[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(GEMM_SMEM)) != cudaSuccess)
             return VELORA_ERR_CUDA;
@@ -304,8 +373,8 @@ int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t
     const int tiles_m = (Mdim + BM - 1) / BM, tiles_n = (Ndim + BN - 1) / BN;
     const int64_t tiles = static_cast<int64_t>(tiles_m) * tiles_n;
     const int grid = static_cast<int>(tiles < di.sm_count ? tiles : di.sm_count);
-    kern<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(ta, tb, static_cast<CT*>(C), ldc, beta, Mdim, Ndim, Kdim,
-                                                   tiles_m, tiles_n, status);
+    kern<<<grid, FUSE ? FUSE_THREADS : GEMM_THREADS, GEMM_SMEM, stream>>>(
+        ta, tb, static_cast<CT*>(C), ldc, beta, Mdim, Ndim, Kdim, tiles_m, tiles_n, status, fz);
     return after_launch();
 }
 
@@ -368,6 +437,23 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
                              void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
                              int dtype, int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream)
 {
+    // Fused path: Dsub a power of two between 8 and 1024 (sub-token boundaries then fall on 16-byte
+    // chunks of the 64-column X tiles); everything else runs the GEMM and the compress kernel in turn.
+    const bool pow2 = Dsub >= 8 && Dsub <= VELORA_MAX_DSUB && (Dsub & (Dsub - 1)) == 0;
+    const bool gemm_ok = dtype == VELORA_BF16 && N >= 1 && N < (1 << 30) && D < (1 << 30) && O < (1 << 30) &&
+                         tc_operand_ok(X, ldx) && tc_operand_ok(W, ldw) && aligned16(Y) && ldy % 8 == 0;
+    if (pow2 && gemm_ok) {
+        CUtensorMap ta, tb;
+        int rc = make_tmap_bf16_2d(&ta, X, D, N, ldx, BK, BM);
+        if (rc != VELORA_OK) return rc;
+        rc = make_tmap_bf16_2d(&tb, W, D, O, ldw, BK, BN);
+        if (rc != VELORA_OK) return rc;
+        FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>(ceil_div64(D, Dsub))};
+        const int m = static_cast<int>(N), n = static_cast<int>(O), k = static_cast<int>(D);
+        if (z_dtype == VELORA_F32)
+            return launch_kernel<false, false, __nv_bfloat16, 1>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);
+        return launch_kernel<false, false, __nv_bfloat16, 2>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);
+    }
     int rc = launch_gemm_tc(GEMM_NT_K_K, X, ldx, W, ldw, Y, dtype, ldy, 0, N, O, D, dtype, status, stream);
     if (rc != VELORA_OK) return rc;
     return launch_compress(X, dtype, N, D, ldx, Dsub, v, Z, z_dtype, ldz, stream);

@@ -71,6 +71,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return true;
 }
 
+// Whole-warp form: lane 0 does the (bounded) waiting, the other lanes then confirm the completed phase
+// with a single probe each, which also gives every lane its own acquire of the data the phase covers.
+// Keeps 31 of 32 lanes from polling shared memory while the tensor cores stream operands out of it.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (ok) {
+        for (int i = 0; i < 1024 && !mbar_try_wait(bar, parity); ++i) {}
+    }
+    return ok != 0;
+}
+
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
