@@ -25,7 +25,8 @@ constexpr int SLAB_BYTES = 64 * BK * 2;           // one 64-wide MN-major slab: 
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int FUSE_THREADS = GEMM_THREADS + 128;    // + four compress warps
-constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256 + VELORA_MAX_DSUB * 4;
+constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256;
+constexpr size_t FUSE_SMEM = GEMM_SMEM + A_BYTES + VELORA_MAX_DSUB * 4;   // + compress tile + copy of v
 
 // Arguments of the compress that rides on the forward GEMM's A tiles (Section 3.1, Eq. 1).
 struct FuseArgs {
@@ -116,12 +117,15 @@ template <> struct Store32<float> {
     }
 };
 
-// FUSE = 0: plain GEMM.  FUSE = 1 / 2 (forward only, A = X K-major): four extra warps read every landed
-// X tile from shared memory and compute Z = compress(X, v) in fp32 / bf16 storage, so X crosses HBM once
-// for both results.  A k-block of 64 columns holds 64/Dsub sub-tokens (or 1/w of one, w = Dsub/64); the
-// CTA working on n-tile j handles the sub-token groups g with g % tiles_n == j, so the work is spread
-// over the CTAs that share a row block.  Thread t of the compress warps owns tile row t; the 128-byte
-// swizzle of the tile makes its 16-byte reads conflict-free.
+// FUSE = 0: plain GEMM.  FUSE = 1 / 2 (forward only, A = X K-major): Z = compress(X, v) (fp32 / bf16
+// storage) is computed by four extra warps from X tiles that are already on their way through L2 for the
+// GEMM, so X crosses HBM once for both results.  A k-block of 64 columns holds 64/Dsub sub-tokens (or
+// 1/w of one, w = Dsub/64); the CTA working on n-tile j handles the sub-token groups g with
+// g % tiles_n == j, so the work is spread over the CTAs that share a row block.  For such a k-block the
+// producer fetches the X tile a second time (an L2 hit) into a buffer of its own with its own pair of
+// barriers: the GEMM ring has no slack to wait for a second reader (four stages barely cover the TMA
+// latency), so the compress warps never touch it.  Thread t of the compress warps owns tile row t; the
+// 128-byte swizzle of the tile makes its 16-byte reads conflict-free.
 template <bool A_MN, bool B_MN, typename CT, int FUSE>
 __global__ void __launch_bounds__(FUSE ? FUSE_THREADS : GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -135,13 +139,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* smem = smem_raw + (base - raw);
     const uint32_t sA = base;
     const uint32_t sB = base + STAGES * A_BYTES;
-    uint8_t* tail = smem + STAGES * (A_BYTES + B_BYTES);
-    const uint32_t bars = base + STAGES * (A_BYTES + B_BYTES);
+    constexpr int CBUF_BYTES = FUSE ? A_BYTES : 0;              // the compress warps' own X tile
+    const uint32_t cbuf = base + STAGES * (A_BYTES + B_BYTES);
+    uint8_t* tail = smem + STAGES * (A_BYTES + B_BYTES) + CBUF_BYTES;
+    const uint32_t bars = cbuf + CBUF_BYTES;
     const uint32_t full = bars, empty = bars + 8 * STAGES;
     const uint32_t tfull = bars + 16 * STAGES, tempty = tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 32);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 40);
+    const uint32_t cfull = tempty + 16, cempty = cfull + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 48);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 56);
     float* sv = reinterpret_cast<float*>(tail + 256);           // copy of v for the compress warps
+    const int cw = (FUSE && fz.Dsub >= BK) ? fz.Dsub / BK : 1;  // k-blocks per sub-token
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -151,12 +159,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full + 8 * s, 1);
-            mbar_init(empty + 8 * s, FUSE ? 5 : 1);             // MMA commit (+ one arrival per compress warp)
+            mbar_init(empty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull + 8 * a, 1);
             mbar_init(tempty + 8 * a, 4);
         }
+        mbar_init(cfull, 1);
+        mbar_init(cempty, 4);                                   // one arrival per compress warp
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
@@ -177,7 +187,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (one lane)
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, oc = 0;
             for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
                 const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -199,10 +209,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         tma_load_2d(sB + s * B_BYTES, &tmB, full + 8 * s, k0, tc0.n0);
                     }
+                    if (FUSE && (kb / cw) % tiles_n == tc0.n0 / BN) {      // this CTA compresses the k-block
+                        if (!mbar_wait(cempty, (oc & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+                        mbar_arrive_expect_tx(cfull, A_BYTES);
+                        tma_load_2d(cbuf, &tmA, cfull, k0, tc0.m0);
+                        ++oc;
+                    }
                 }
             }
             if (failed) {
                 *abort_flag = 1;
+                if (FUSE && oc > 0) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(cfull, (oc - 1u) & 1u))
+                        if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+                }
                 // Let this CTA's own copies in flight land before shared memory is given up.
                 const uint32_t back = it < STAGES ? it : STAGES;
                 for (uint32_t j = 1; j <= back; ++j) {
@@ -249,49 +270,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------ compress (4 warps, one tile row per thread)
         const int trow = (warp - 6) * 32 + lane;
         const int Dsub = fz.Dsub;
-        const int w = Dsub >= BK ? Dsub / BK : 1;              // k-blocks per sub-token
         const int nsub = Dsub >= BK ? 1 : BK / Dsub;           // sub-tokens per k-block
+        const uint32_t rowaddr = cbuf + trow * 128;
         float acc = 0.f;
-        uint32_t it = 0;
+        uint32_t oc = 0;
         for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
             const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
             const int tn = tc0.n0 / BN;
             const int row = tc0.m0 + trow;
-            for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                if (!mbar_wait_warp(full + 8 * s, ph, abort_flag)) { failed = true; break; }
-                const int g = kb / w;
-                if (g % tiles_n == tn) {
-                    const uint32_t rowaddr = sA + s * A_BYTES + trow * 128;
-                    const int j0 = (kb % w) * BK;              // position of this k-block inside the sub-token
-                    if (kb % w == 0) acc = 0.f;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if ((kb / cw) % tiles_n != tn) continue;
+                if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
+                ++oc;
+                uint4 d[8];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint4 d;
-                        const uint32_t a = rowaddr + (static_cast<uint32_t>(c ^ (trow & 7)) << 4);
-                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(d.x), "=r"(d.y), "=r"(d.z), "=r"(d.w) : "r"(a));
-                        const int jv = (j0 + c * 8) % Dsub;    // Dsub and 8 are powers of two here
-                        const float4 va = *reinterpret_cast<const float4*>(sv + jv);
-                        const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
-                        if (nsub > 1 && jv == 0) acc = 0.f;    // a new sub-token starts inside the k-block
-                        acc = fmaf(bf16_lo(d.x), va.x, acc); acc = fmaf(bf16_hi(d.x), va.y, acc);
-                        acc = fmaf(bf16_lo(d.y), va.z, acc); acc = fmaf(bf16_hi(d.y), va.w, acc);
-                        acc = fmaf(bf16_lo(d.z), vb.x, acc); acc = fmaf(bf16_hi(d.z), vb.y, acc);
-                        acc = fmaf(bf16_lo(d.w), vb.z, acc); acc = fmaf(bf16_hi(d.w), vb.w, acc);
-                        // The sub-token ends with this chunk, or the row does (ragged last sub-token: the
-                        // columns beyond D were zero-filled by TMA and no further k-block follows).
-                        if (jv + 8 == Dsub || (kb == kblocks - 1 && c == 7)) {
-                            const int m = (kb * BK + c * 8) / Dsub;
-                            if (row < Mdim && m < fz.M) {
-                                if (FUSE == 1) static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = acc;
-                                else static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
-                            }
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t a = rowaddr + (static_cast<uint32_t>(c ^ (trow & 7)) << 4);
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(d[c].x), "=r"(d[c].y), "=r"(d[c].z), "=r"(d[c].w) : "r"(a));
+                }
+                const int j0 = (kb % cw) * BK;                 // position of this k-block inside the sub-token
+                if (kb % cw == 0) acc = 0.f;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const int jv = (j0 + c * 8) & (Dsub - 1);  // Dsub is a power of two here
+                    const float4 va = *reinterpret_cast<const float4*>(sv + jv);
+                    const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
+                    if (nsub > 1 && jv == 0) acc = 0.f;        // a new sub-token starts inside the k-block
+                    float a0 = bf16_lo(d[c].x) * va.x, a1 = bf16_hi(d[c].x) * va.y;
+                    a0 = fmaf(bf16_lo(d[c].y), va.z, a0); a1 = fmaf(bf16_hi(d[c].y), va.w, a1);
+                    a0 = fmaf(bf16_lo(d[c].z), vb.x, a0); a1 = fmaf(bf16_hi(d[c].z), vb.y, a1);
+                    a0 = fmaf(bf16_lo(d[c].w), vb.z, a0); a1 = fmaf(bf16_hi(d[c].w), vb.w, a1);
+                    acc += a0 + a1;
+                    // The sub-token ends with this chunk, or the row does (ragged last sub-token: the
+                    // columns beyond D were zero-filled by TMA and no further k-block follows).
+                    if (jv + 8 == Dsub || (kb == kblocks - 1 && c == 7)) {
+                        const int m = (kb * BK + c * 8) / Dsub;
+                        if (row < Mdim && m < fz.M) {
+                            if (FUSE == 1) static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = acc;
+                            else static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty + 8 * s);     // this warp is done with the stage
+                __syncwarp();                                  // every lane's reads of the tile are done
+                if (lane == 0) mbar_arrive(cempty);
             }
         }
         if (failed) *abort_flag = 1;
@@ -302,7 +324,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x, ++t) {
             const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
             const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
-            if (!mbar_wait_warp(tfull + 8 * acc, aph, abort_flag)) { failed = true; break; }
+            if (!mbar_wait_warp(tfull + 8 * acc, aph, abort_flag, 256)) { failed = true; break; }
             tc_fence_after_sync();
             const int row = tc0.m0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + acc * BN + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -363,7 +385,8 @@ int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
     auto kern = gemm_tc_kernel<A_MN, B_MN, CT, FUSE>;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(GEMM_SMEM)) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(FUSE ? FUSE_SMEM : GEMM_SMEM)) != cudaSuccess)
             return VELORA_ERR_CUDA;
         configured[dev] = true;
     }
@@ -373,7 +396,7 @@ int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t
     const int tiles_m = (Mdim + BM - 1) / BM, tiles_n = (Ndim + BN - 1) / BN;
     const int64_t tiles = static_cast<int64_t>(tiles_m) * tiles_n;
     const int grid = static_cast<int>(tiles < di.sm_count ? tiles : di.sm_count);
-    kern<<<grid, FUSE ? FUSE_THREADS : GEMM_THREADS, GEMM_SMEM, stream>>>(
+    kern<<<grid, FUSE ? FUSE_THREADS : GEMM_THREADS, FUSE ? FUSE_SMEM : GEMM_SMEM, stream>>>(
         ta, tb, static_cast<CT*>(C), ldc, beta, Mdim, Ndim, Kdim, tiles_m, tiles_n, status, fz);
     return after_launch();
 }
@@ -442,7 +465,10 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
     const bool pow2 = Dsub >= 8 && Dsub <= VELORA_MAX_DSUB && (Dsub & (Dsub - 1)) == 0;
     const bool gemm_ok = dtype == VELORA_BF16 && N >= 1 && N < (1 << 30) && D < (1 << 30) && O < (1 << 30) &&
                          tc_operand_ok(X, ldx) && tc_operand_ok(W, ldw) && aligned16(Y) && ldy % 8 == 0;
-    if (pow2 && gemm_ok) {
+    // One CTA compresses one k-block in tiles_n; with fewer than four n-tiles the compress warps would
+    // hold the producer back, so narrow outputs take the two-kernel route as well.
+    const bool wide = (O + BN - 1) / BN >= 4;
+    if (pow2 && gemm_ok && wide) {
         CUtensorMap ta, tb;
         int rc = make_tmap_bf16_2d(&ta, X, D, N, ldx, BK, BM);
         if (rc != VELORA_OK) return rc;

@@ -57,13 +57,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Waits for the phase with the given parity to complete.  Never spins for ever: returns false when
 // another role has raised `abort_flag` or after kWaitLimitNs; the caller then raises the flag itself,
 // records the failure and leaves its loop.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t backoff_ns = 0)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 63u) == 0u) {
+        // Waiters off the critical path sleep between probes: a tight probe loop costs issue slots and
+        // shared-memory bandwidth that the tensor cores' operand stream needs.
+        if (backoff_ns) __nanosleep(backoff_ns);
+        if ((++spins & 63u) == 0u || backoff_ns) {
             if (*abort_flag) return false;
             if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
         }
@@ -74,10 +78,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // Whole-warp form: lane 0 does the (bounded) waiting, the other lanes then confirm the completed phase
 // with a single probe each, which also gives every lane its own acquire of the data the phase covers.
 // Keeps 31 of 32 lanes from polling shared memory while the tensor cores stream operands out of it.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               uint32_t backoff_ns = 0)
 {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, backoff_ns) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (ok) {
         for (int i = 0; i < 1024 && !mbar_try_wait(bar, parity); ++i) {}
