@@ -5,17 +5,23 @@
 // once); the contraction over tokens is small next to it and runs on tcgen05 so that it hides under
 // the dY stream.
 //
-// Three launches:
-//   1. z_to_bf16_kernel   Z (fp32 or bf16, any pitch) -> Zb[N, pitch] bf16, pitch = round_up(M, 64),
-//                         zero padded, so that TMA can fetch 64-wide MN-major slabs.
-//   2. wg_partial_kernel  grid (O/128, splits): CTA (t, s) multiplies dY[:, 128t : 128t+128]^T with Zb
-//                         over its share of the tokens.  Both operands are MN-major (tokens are the K
-//                         dimension and rows of dY / Zb are tokens): 64 x 64 TMA boxes, MN-major
-//                         matrix descriptors, no transpose.  fp32 accumulator in TMEM, written as a
-//                         partial product P[s][o][m].
-//   3. expand_p kernel    sums the partials in fixed order and streams dW = P (x) v over all SMs.
-// Splitting the token range keeps every SM pulling on dY; summing partials in a fixed order keeps the
-// result run-to-run identical.
+//   z_to_bf16_kernel   Z (fp32 or bf16, any pitch) -> Zb[N, pitch] bf16, pitch = round_up(M, 64), zero
+//                      padded, so that TMA can fetch 64-wide MN-major slabs.
+//   wg_kernel          grid (O/128, S): CTA (t, s) multiplies dY[:, 128t : 128t+128]^T with Zb over its
+//                      share of the tokens.  Both operands are MN-major (tokens are the K dimension and
+//                      rows of dY / Zb are tokens): 64 x 64 TMA boxes, MN-major matrix descriptors, no
+//                      transpose; fp32 accumulator in TMEM.  Splitting the token range keeps every SM
+//                      pulling on dY.
+//     CLUSTER = true   the S CTAs of an output tile form a thread-block cluster.  Each parks its partial
+//                      product in its own shared memory; after a cluster barrier CTA s adds the S
+//                      partials of its share of the 128 rows through distributed shared memory, in a
+//                      fixed order, and streams dW = P (x) v for those rows.  One launch, no partials in
+//                      global memory, every SM takes part in the write.
+//     CLUSTER = false  the partials go to the workspace and launch_expand_p sums and expands them
+//                      (shapes the cluster form does not take: Dsub not 8 * 2^k, unaligned dW rows).
+// Summing the partials in a fixed order keeps the result run-to-run identical.
+#include <cooperative_groups.h>
+
 #include "gemm_tc.cuh"
 #include "tc_common.cuh"
 
@@ -29,7 +35,7 @@ constexpr int WG_BM = 128, WG_BK = 64, WG_STAGES = 4;
 constexpr int WG_A_BYTES = WG_BM * WG_BK * 2;         // 16 KB: two 64-wide slabs of dY^T
 constexpr int WG_SLAB = 64 * WG_BK * 2;               // 8 KB
 constexpr int WG_THREADS = 192;
-constexpr int WG_MAX_SPLITS = 8;
+constexpr int WG_MAX_SPLITS = 8;                      // also the portable cluster size limit
 constexpr int WG_MAX_M = 256;
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
@@ -56,16 +62,71 @@ z_to_bf16_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int M, int pi
     }
 }
 
+struct WgArgs {
+    float* partials;          // CLUSTER = false: [S][O][ldp]
+    int64_t split_stride;
+    int O, n_slabs, npad, tmem_cols, kblocks, kb_per_split, ldp;
+    int* status;
+    // CLUSTER = true: the expansion
+    const float* v;
+    void* dW;
+    int64_t lddw;
+    int D, M, beta, splits;
+};
+
+template <typename WT> struct WgOut8;
+template <> struct WgOut8<__nv_bfloat16> {
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, float (&y)[8], int beta)
+    {
+        uint4* q = reinterpret_cast<uint4*>(p);
+        if (beta) {
+            const uint4 old = *q;
+            y[0] += bf16_lo(old.x); y[1] += bf16_hi(old.x);
+            y[2] += bf16_lo(old.y); y[3] += bf16_hi(old.y);
+            y[4] += bf16_lo(old.z); y[5] += bf16_hi(old.z);
+            y[6] += bf16_lo(old.w); y[7] += bf16_hi(old.w);
+        }
+        uint4 o;
+        o.x = pack_bf16x2(y[0], y[1]);
+        o.y = pack_bf16x2(y[2], y[3]);
+        o.z = pack_bf16x2(y[4], y[5]);
+        o.w = pack_bf16x2(y[6], y[7]);
+        __stcs(q, o);
+    }
+};
+template <> struct WgOut8<float> {
+    static __device__ __forceinline__ void store(float* p, float (&y)[8], int beta)
+    {
+        float4* q = reinterpret_cast<float4*>(p);
+        if (beta) {
+            const float4 a = q[0], b = q[1];
+            y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
+            y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
+        }
+        __stcs(q, make_float4(y[0], y[1], y[2], y[3]));
+        __stcs(q + 1, make_float4(y[4], y[5], y[6], y[7]));
+    }
+};
+
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t remote;
+    float x;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x) : "r"(remote) : "memory");
+    return x;
+}
+
+// LPS, CH, WT describe the expansion (CLUSTER = true only): Dsub = 8 * LPS * CH, dW element type.
+template <bool CLUSTER, int LPS, int CH, typename WT>
 __global__ void __launch_bounds__(WG_THREADS, 2)
-wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmZ,
-                  float* __restrict__ partials, int O, int n_slabs, int npad, int tmem_cols,
-                  int kblocks, int kb_per_split, int64_t split_stride, int ldp, int* __restrict__ status)
+wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmZ, const WgArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const int stage_bytes = WG_A_BYTES + n_slabs * WG_SLAB;
+    const int stage_bytes = WG_A_BYTES + a.n_slabs * WG_SLAB;
     uint8_t* tail = smem + WG_STAGES * stage_bytes;
     const uint32_t bars = base + WG_STAGES * stage_bytes;
     const uint32_t full = bars, empty = bars + 8 * WG_STAGES, tfull = bars + 16 * WG_STAGES;
@@ -74,9 +135,9 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int o0 = blockIdx.x * WG_BM;
-    const int split = blockIdx.y;
-    const int kb0 = split * kb_per_split;
-    const int kb1 = (kb0 + kb_per_split < kblocks) ? kb0 + kb_per_split : kblocks;
+    const int split = blockIdx.y;                            // = rank in the cluster when CLUSTER
+    const int kb0 = split * a.kb_per_split;
+    const int kb1 = (kb0 + a.kb_per_split < a.kblocks) ? kb0 + a.kb_per_split : a.kblocks;
     const int nkb = kb1 - kb0;                               // >= 1 by construction on the host
 
     if (threadIdx.x == 0) {
@@ -91,13 +152,17 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
         prefetch_tensormap(&tmZ);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), static_cast<uint32_t>(tmem_cols));
+        tmem_alloc(smem_u32(tmem_slot), static_cast<uint32_t>(a.tmem_cols));
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+
+    // Partial product of this CTA in its own shared memory (CLUSTER): rows of ldsp floats over the ring,
+    // which is idle once the accumulator is complete.
+    const int ldsp = a.npad + 4;
 
     bool failed = false;
     if (warp == 0) {
@@ -111,7 +176,7 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
                 const uint32_t a_dst = base + s * stage_bytes;
                 tma_load_2d(a_dst, &tmY, full + 8 * s, o0, k0);
                 tma_load_2d(a_dst + WG_SLAB, &tmY, full + 8 * s, o0 + 64, k0);
-                for (int i = 0; i < n_slabs; ++i)
+                for (int i = 0; i < a.n_slabs; ++i)
                     tma_load_2d(a_dst + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * s, 64 * i, k0);
             }
             if (failed) {
@@ -127,7 +192,7 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(WG_BM, npad, true, true);
+            const uint32_t idesc = umma_idesc_bf16(WG_BM, a.npad, true, true);
             for (int it = 0; it < nkb; ++it) {
                 const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
                 if (!mbar_wait(full + 8 * s, ph, abort_flag)) { failed = true; break; }
@@ -146,22 +211,24 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
         }
     } else {
         const int quarter = warp & 3;
-        if (!mbar_wait(tfull, 0u, abort_flag)) {
+        if (!mbar_wait_warp(tfull, 0u, abort_flag, 256)) {
             failed = true;
             *abort_flag = 1;
         } else {
             tc_fence_after_sync();
-            const int o = o0 + quarter * 32 + lane;
+            const int trow = quarter * 32 + lane;
+            const int o = o0 + trow;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            float* prow = partials + split * split_stride + static_cast<int64_t>(o) * ldp;
-            for (int c = 0; c * 32 < npad; ++c) {
+            float* prow = CLUSTER ? reinterpret_cast<float*>(smem) + trow * ldsp
+                                  : a.partials + split * a.split_stride + static_cast<int64_t>(o) * a.ldp;
+            for (int c = 0; c * 32 < a.npad; ++c) {
                 uint32_t r[32];
                 tmem_ld_32x32(taddr + c * 32, r);
                 tmem_ld_wait();
-                if (o < O) {
+                if (CLUSTER || o < a.O) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if (c * 32 + 4 * i < npad)                 // npad is a multiple of 16
+                        if (c * 32 + 4 * i < a.npad)               // npad is a multiple of 16
                             *reinterpret_cast<float4*>(prow + c * 32 + 4 * i) =
                                 make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
                                             __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
@@ -169,14 +236,74 @@ wg_partial_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant
             }
         }
     }
-    if (failed && status) atomicExch(status, VELORA_ERR_TIMEOUT);
+    if (failed && a.status) atomicExch(a.status, VELORA_ERR_TIMEOUT);
 
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     if (warp == 1) {
         __syncwarp();
-        tmem_dealloc(tmem_base, static_cast<uint32_t>(tmem_cols));
+        tmem_dealloc(tmem_base, static_cast<uint32_t>(a.tmem_cols));
+    }
+
+    if (CLUSTER) {
+        // Every CTA reaches both cluster barriers whatever happened above (a timed-out role only skips
+        // its own loop), so the cluster cannot deadlock on a CTA that gave up.
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();                                      // all partials of the tile are in shared memory
+
+        constexpr int L = LPS * CH;
+        constexpr int SPW = 32 / LPS;
+        const int q = lane & (LPS - 1), sub = lane / LPS;
+        float vr[CH][8];
+#pragma unroll
+        for (int i = 0; i < CH; ++i)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(a.v + 8 * (q + LPS * i) + e);
+
+        const int rows_per = (WG_BM + a.splits - 1) / a.splits;
+        const int r_begin = split * rows_per;
+        const int r_end = (r_begin + rows_per < WG_BM) ? r_begin + rows_per : WG_BM;
+        WT* dW = static_cast<WT*>(a.dW);
+        for (int trow = r_begin + warp; trow < r_end; trow += WG_THREADS / 32) {
+            const int o = o0 + trow;
+            if (o >= a.O) break;
+            for (int m0 = 0; m0 < a.M; m0 += 32) {
+                float p = 0.f;
+                if (m0 + lane < a.M) {
+                    const uint32_t laddr = base + static_cast<uint32_t>((trow * ldsp + m0 + lane) * 4);
+                    for (int s = 0; s < a.splits; ++s) p += ld_cluster_f32(laddr, static_cast<uint32_t>(s));   // fixed order
+                }
+                WT* ptr = dW + static_cast<int64_t>(o) * a.lddw + (static_cast<int64_t>(m0 + sub) * L + q) * 8;
+#pragma unroll 8
+                for (int it = 0; it < LPS; ++it, ptr += SPW * L * 8) {
+                    const int ms = it * SPW + sub;
+                    const float pm = __shfl_sync(0xffffffffu, p, ms);
+                    if (m0 + ms >= a.M) continue;
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) {
+                        const int col = ((m0 + ms) * L + q + LPS * i) * 8;
+                        float y[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) y[e] = pm * vr[i][e];
+                        if (col + 8 <= a.D) {
+                            WgOut8<WT>::store(ptr + i * LPS * 8, y, a.beta);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                if (col + e < a.D) {
+                                    WT* pe = ptr + i * LPS * 8 + e;
+                                    float f = y[e];
+                                    if (a.beta) f += Elem<WT>::load(pe);
+                                    Elem<WT>::store(pe, f);
+                                }
+                        }
+                    }
+                }
+            }
+        }
+        cluster.sync();                                      // nobody leaves while its partial is still being read
     }
 }
 
@@ -216,6 +343,38 @@ WgPlan make_plan(int64_t N, int64_t D, int64_t O, int Dsub, int sm_count)
     p.part_bytes = static_cast<size_t>(WG_MAX_SPLITS) * static_cast<size_t>(O) * p.npad * sizeof(float);
     p.ok = true;
     return p;
+}
+
+template <bool CLUSTER, int LPS, int CH, typename WT>
+int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, const WgPlan& p, int smem_optin,
+              cudaStream_t stream)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
+    auto kern = wg_kernel<CLUSTER, LPS, CH, WT>;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
+            return VELORA_ERR_CUDA;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(p.tiles_o), static_cast<unsigned>(p.splits), 1);
+    cfg.blockDim = dim3(WG_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = p.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = CLUSTER ? static_cast<unsigned>(p.splits) : 1u;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tmY, tmZ, a) != cudaSuccess) {
+        cudaGetLastError();
+        return VELORA_ERR_CUDA;
+    }
+    return after_launch();
 }
 
 }  // namespace
@@ -260,31 +419,59 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
         rc = after_launch();
         if (rc != VELORA_OK) return rc;
     }
-    // 2. partial products on the tensor cores
-    {
-        CUtensorMap tmY, tmZ;
-        rc = make_tmap_bf16_2d(&tmY, dY, O, N, lddy, 64, WG_BK);
-        if (rc != VELORA_OK) return rc;
-        rc = make_tmap_bf16_2d(&tmZ, Zb, p.pitch, N, p.pitch, 64, WG_BK);
-        if (rc != VELORA_OK) return rc;
-        static bool configured[64] = {};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
-        if (!configured[dev]) {
-            if (cudaFuncSetAttribute(wg_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     di.smem_optin) != cudaSuccess)
-                return VELORA_ERR_CUDA;
-            configured[dev] = true;
-        }
-        const int64_t split_stride = static_cast<int64_t>(O) * p.npad;
-        dim3 grid(static_cast<unsigned>(p.tiles_o), static_cast<unsigned>(p.splits));
-        wg_partial_kernel<<<grid, WG_THREADS, p.smem, stream>>>(tmY, tmZ, partials, static_cast<int>(O), p.n_slabs,
-                                                               p.npad, p.tmem_cols, p.kblocks, p.kb_per_split,
-                                                               split_stride, p.npad, status);
-        rc = after_launch();
-        if (rc != VELORA_OK) return rc;
+
+    CUtensorMap tmY, tmZ;
+    rc = make_tmap_bf16_2d(&tmY, dY, O, N, lddy, 64, WG_BK);
+    if (rc != VELORA_OK) return rc;
+    rc = make_tmap_bf16_2d(&tmZ, Zb, p.pitch, N, p.pitch, 64, WG_BK);
+    if (rc != VELORA_OK) return rc;
+
+    WgArgs a{};
+    a.partials = partials;
+    a.split_stride = static_cast<int64_t>(O) * p.npad;
+    a.O = static_cast<int>(O);
+    a.n_slabs = p.n_slabs;
+    a.npad = p.npad;
+    a.tmem_cols = p.tmem_cols;
+    a.kblocks = p.kblocks;
+    a.kb_per_split = p.kb_per_split;
+    a.ldp = p.npad;
+    a.status = status;
+    a.v = v;
+    a.dW = dW;
+    a.lddw = lddw;
+    a.D = static_cast<int>(D);
+    a.M = p.M;
+    a.beta = beta;
+    a.splits = p.splits;
+
+    // 2a. one launch: cluster of the tile's splits, reduction through distributed shared memory
+    const int L = (Dsub % 8 == 0) ? Dsub / 8 : 0;
+    const bool vec = L >= 1 && L <= 128 && (L & (L - 1)) == 0 && aligned16(dW) &&
+                     (lddw * static_cast<int64_t>(dtype_size(dw_dtype))) % 16 == 0 &&
+                     static_cast<size_t>(WG_BM) * (p.npad + 4) * 4 <= static_cast<size_t>(WG_STAGES) * (WG_A_BYTES + p.n_slabs * WG_SLAB);
+    if (vec) {
+        const int lps = L < 32 ? L : 32, ch = L / lps;
+        rc = VELORA_ERR_CUDA;
+#define VELORA_WG_CASE(LPSV, CHV)                                                                             \
+        if (lps == LPSV && ch == CHV)                                                                         \
+            rc = dw_dtype == VELORA_BF16                                                                      \
+                     ? launch_wg<true, LPSV, CHV, __nv_bfloat16>(tmY, tmZ, a, p, di.smem_optin, stream)       \
+                     : launch_wg<true, LPSV, CHV, float>(tmY, tmZ, a, p, di.smem_optin, stream)
+        VELORA_WG_CASE(1, 1);
+        VELORA_WG_CASE(2, 1);
+        VELORA_WG_CASE(4, 1);
+        VELORA_WG_CASE(8, 1);
+        VELORA_WG_CASE(16, 1);
+        VELORA_WG_CASE(32, 1);
+        VELORA_WG_CASE(32, 2);
+        VELORA_WG_CASE(32, 4);
+#undef VELORA_WG_CASE
+        if (rc == VELORA_OK) return rc;          // a refused cluster launch falls through to the three-launch route
     }
-    // 3. dW = (sum of partials) (x) v
+    // 2b. partial products to the workspace, then 3. dW = (sum of partials) (x) v
+    rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, p, di.smem_optin, stream);
+    if (rc != VELORA_OK) return rc;
     return launch_expand_p(partials, p.splits, static_cast<int64_t>(O) * p.npad, p.npad, v, O, D, Dsub,
                            dW, dw_dtype, lddw, beta, stream);
 }
