@@ -155,6 +155,52 @@ def test_edge_shapes_all_entry_points(vl, N, D, O, Dsub, dtype):
     assert_matches(dW, dW_ref, TOL_GEMM, "dW")
 
 
+FUSED_EDGE = [
+    # N, D, O, Dsub: outputs wide enough (>= 4 column tiles) for the forward to compute Z inside the GEMM
+    (300, 320, 1100, 16),    # four sub-tokens per 64-column block
+    (200, 264, 1024, 8),     # eight per block; D not a multiple of 64
+    (257, 1376, 1040, 64),   # ragged last sub-token (32 of 64 columns)
+    (130, 320, 1025, 256),   # sub-token spans four blocks, the last one has only one block of columns
+    (513, 640, 1536, 128),   # sub-token spans two blocks
+    (129, 2048, 1030, 1024), # longest sub-token
+]
+
+
+@pytest.mark.parametrize("N,D,O,Dsub", FUSED_EDGE)
+@pytest.mark.parametrize("z_dtype", [torch.float32, torch.bfloat16])
+def test_forward_with_compress_inside_the_gemm(vl, N, D, O, Dsub, z_dtype):
+    case = vi.small_case(9000 + D + Dsub, N, D, O, dtype="bf16", mean_offset=0.25)
+    Xa, Wa = case["X"], case["W"]
+    X, W = Xa.torch(DEV), Wa.torch(DEV)
+    v = vl.velora_init_v(X, Dsub)
+    v64 = to_f64(v)
+    ws = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_LINEAR_FORWARD, N, D, O, Dsub), DEV)
+    Y, Z = vl.velora_linear_forward(X, W, v, z_dtype=z_dtype, ws=ws)
+    assert vl.velora_workspace_status(ws) == 0
+    assert_matches(Y, oracle.linear_forward(Xa.f64(), Wa.f64()), TOL_GEMM, "Y")
+    assert_matches(Z, oracle.compress(Xa.f64(), v64), TOL_Z, "Z", ulps=1 if z_dtype == torch.bfloat16 else None)
+    # the stand-alone kernel and the fused path agree to fp32 rounding
+    assert rel_err(to_f64(Z), to_f64(vl.velora_compress(X, v, z_dtype=z_dtype))) < (4e-3 if z_dtype == torch.bfloat16 else 1e-5)
+    assert vl.velora_device_error() == 0
+
+
+def test_no_device_wait_expired_during_a_full_layer(vl):
+    cfg = vi.CONFIGS[3]
+    li = 0
+    X, W, dY = vi.make_X(cfg, li).torch(DEV), vi.make_W(cfg, li).torch(DEV), vi.make_dY(cfg, li).torch(DEV)
+    N, D = X.shape
+    O = W.shape[0]
+    ws = vl.velora_workspace_alloc(max(vl.velora_workspace_bytes(op, N, D, O, 32) for op in
+                                       (vl.OP_INIT_V, vl.OP_LINEAR_BACKWARD_FACTORED, vl.OP_LINEAR_BACKWARD_EXPLICIT)), DEV)
+    v = vl.velora_init_v(X, 32, ws=ws)
+    Y, Z = vl.velora_linear_forward(X, W, v, ws=ws)
+    for mode in (vl.WG_FACTORED, vl.WG_EXPLICIT):
+        vl.velora_linear_backward(dY, W, Z, v, mode=mode, ws=ws)
+    vl.velora_compress(X, v)
+    assert vl.velora_workspace_status(ws) == 0
+    assert vl.velora_device_error() == 0
+
+
 def test_gradient_accumulation_beta_one(vl):
     case = vi.small_case(11, 200, 256, 96, dtype="bf16")
     X, dY = case["X"].torch(DEV), case["dY"].torch(DEV)
