@@ -205,6 +205,33 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
                            void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The two halves of velora_init_v, for a batch that is sharded over several processes (Section 3.2:
+ * the average runs over ALL sub-tokens of the first batch, so every rank must end up with the same v).
+ *   velora_subtoken_sum:  s[j] = sum_n sum_m X[n, m*Dsub + j]   (fp32, s[Dsub]; asynchronous; N == 0 gives 0)
+ *   velora_normalize_v:   v = s / ||s||_2; synchronises `stream`; VELORA_ERR_DEGENERATE_V as velora_init_v
+ * Between the two the caller adds the s of all ranks (an all-reduce of Dsub floats).
+ * ws: velora_workspace_bytes(VELORA_OP_INIT_V, ...) bytes for the sum, at least 256 bytes for the normalisation.
+ */
+int velora_subtoken_sum(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                        float* s, void* ws, size_t ws_bytes, void* stream);
+int velora_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The factored weight gradient kept in factored form (the rank-1 structure of Section 3.2, per sub-token):
+ *   velora_weight_grad_p:  P[O, M] = beta * P + dY^T Z      (fp32, ldp >= M)
+ *   velora_expand_p:       dW[o, m*Dsub + j] = beta * dW + P[o, m] * v[j]
+ * Since v is frozen, P can be accumulated over micro-batches (beta = 1) and summed over data-parallel
+ * ranks (an all-reduce of O*M floats instead of O*D gradients) before it is expanded ONCE; the two calls in
+ * sequence give the same dW as velora_weight_grad in VELORA_WG_FACTORED mode.
+ * ws of velora_weight_grad_p: velora_workspace_bytes(VELORA_OP_WEIGHT_GRAD_FACTORED, N, D, O, Dsub).
+ */
+int velora_weight_grad_p(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                         const void* Z, int z_dtype, int64_t ldz, int64_t D, int Dsub,
+                         float* P, int64_t ldp, int beta, void* ws, size_t ws_bytes, void* stream);
+int velora_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
+                    void* dW, int dw_dtype, int64_t lddw, int beta, void* stream);
+
+/*
  * One forward + backward of a VeLoRA linear (Algorithm 1, both functions) on data
  * that lives in HOST memory (bf16, dense rows: ld = width).  On `stream`, in order:
  * copies X[N, D] and dY[N, O] from the host into the device staging area, runs

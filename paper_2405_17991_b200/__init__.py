@@ -10,7 +10,8 @@ from .binding import (  # noqa: F401
     WG_FACTORED, VeloraError, lib, num_subtokens, velora_compress, velora_init_v, velora_init_v_static,
     velora_linear_backward, velora_linear_forward, velora_reconstruct, velora_status_string,
     velora_version, velora_weight_grad, velora_workspace_alloc, velora_workspace_bytes,
-    velora_workspace_init, velora_workspace_status, velora_launch_count, velora_device_error,
+    velora_workspace_init, velora_workspace_status, velora_launch_count, velora_device_error, velora_subtoken_sum, velora_normalize_v,
+    velora_weight_grad_p, velora_expand_p,
     velora_host_step_staging_bytes, velora_linear_step_host,
 )
 from .memory_model import saved_activation_bytes  # noqa: F401

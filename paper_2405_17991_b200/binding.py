@@ -37,6 +37,10 @@ SIGNATURES = {
     "velora_device_error": (_int, [_p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
     "velora_init_v_static": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p]),
+    "velora_subtoken_sum": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
+    "velora_normalize_v": (_int, [_p, _int, _p, _p, _sz, _p]),
+    "velora_weight_grad_p": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _i64, _int, _p, _i64, _int, _p, _sz, _p]),
+    "velora_expand_p": (_int, [_p, _i64, _p, _i64, _i64, _int, _p, _int, _i64, _int, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_reconstruct": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_weight_grad": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _p, _i64, _int,
@@ -306,3 +310,59 @@ def velora_linear_step_host(hX: torch.Tensor, hdY: torch.Tensor, W: torch.Tensor
         ctypes.c_void_p(staging.data_ptr()), staging.numel(), N, D, O, Dsub,
         ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
     _check(rc, "velora_linear_step_host")
+
+
+def velora_subtoken_sum(X: torch.Tensor, Dsub: int, s: Optional[torch.Tensor] = None,
+                        ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Un-normalised sub-token sum of this rank's shard (add the ranks' sums, then velora_normalize_v)."""
+    N, D = X.shape
+    xp, ldx = (_mat(X, "X") if N > 0 else (ctypes.c_void_p(0), D))
+    if s is None:
+        s = torch.empty(Dsub, dtype=torch.float32, device=X.device)
+    ws = _ws(ws, velora_workspace_bytes(OP_INIT_V, max(N, 1), D, 1, Dsub), X.device)
+    rc = lib().velora_subtoken_sum(xp, _dt(X), N, D, ldx, Dsub, _vec(s), ctypes.c_void_p(ws.data_ptr()), ws.numel(),
+                                   _stream(stream))
+    _check(rc, "velora_subtoken_sum")
+    return s
+
+
+def velora_normalize_v(s: torch.Tensor, v: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                       stream=None) -> torch.Tensor:
+    Dsub = s.shape[0]
+    if v is None:
+        v = torch.empty_like(s)
+    ws = _ws(ws, 256, s.device)
+    rc = lib().velora_normalize_v(_vec(s), Dsub, _vec(v), ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_normalize_v")
+    return v
+
+
+def velora_weight_grad_p(dY: torch.Tensor, Z: torch.Tensor, D: int, Dsub: int, P: Optional[torch.Tensor] = None,
+                         beta: int = 0, ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """P[O, M] = beta * P + dY^T Z in fp32: the weight gradient before its expansion by v."""
+    N, O = dY.shape
+    M = num_subtokens(D, Dsub)
+    yp, lddy = (_mat(dY, "dY") if N > 0 else (ctypes.c_void_p(0), O))
+    zp, ldz = (_mat(Z, "Z") if N > 0 else (ctypes.c_void_p(0), M))
+    if P is None:
+        P = torch.zeros((O, M), dtype=torch.float32, device=dY.device)
+    pp, ldp = _mat(P, "P")
+    ws = _ws(ws, velora_workspace_bytes(OP_WEIGHT_GRAD_FACTORED, N, D, O, Dsub), dY.device)
+    rc = lib().velora_weight_grad_p(yp, _dt(dY), N, O, lddy, zp, _dt(Z), ldz, D, Dsub, pp, ldp, beta,
+                                    ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_weight_grad_p")
+    return P
+
+
+def velora_expand_p(P: torch.Tensor, v: torch.Tensor, D: int, dW: Optional[torch.Tensor] = None,
+                    dw_dtype=torch.bfloat16, beta: int = 0, stream=None) -> torch.Tensor:
+    """dW[o, m*Dsub + j] = beta * dW + P[o, m] v[j]."""
+    O = P.shape[0]
+    Dsub = v.shape[0]
+    pp, ldp = _mat(P, "P")
+    if dW is None:
+        dW = torch.empty((O, D), dtype=dw_dtype, device=P.device)
+    wp, lddw = _mat(dW, "dW")
+    rc = lib().velora_expand_p(pp, ldp, _vec(v), O, D, Dsub, wp, _dt(dW), lddw, beta, _stream(stream))
+    _check(rc, "velora_expand_p")
+    return dW

@@ -353,4 +353,75 @@ int velora_linear_step_host(const void* hX, const void* hdY, void* hY, void* hdX
     return VELORA_OK;
 }
 
+int velora_subtoken_sum(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                        float* s, void* ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!s) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(s, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (N == 0)                                           /* an empty shard contributes a zero sum */
+        return cudaMemsetAsync(s, 0, sizeof(float) * Dsub, st) == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    if (!X) return VELORA_ERR_INVALID_ARG;
+    if (ldx < D) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(X, x_dtype)) return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return launch_init_v(X, x_dtype, N, D, ldx, Dsub, s, ws, ws_bytes, st, 1);
+}
+
+int velora_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!s || !v || Dsub < 1) return VELORA_ERR_INVALID_ARG;
+    if (Dsub > VELORA_MAX_DSUB) return VELORA_ERR_UNSUPPORTED;
+    if (!elem_aligned(s, VELORA_F32) || !elem_aligned(v, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return launch_normalize_v(s, Dsub, v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int velora_weight_grad_p(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                         const void* Z, int z_dtype, int64_t ldz, int64_t D, int Dsub,
+                         float* P, int64_t ldp, int beta, void* ws, size_t ws_bytes, void* stream)
+{
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(dy_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    const int64_t M = num_subtokens(D, Dsub);
+    if (!P || ldp < M || (beta != 0 && beta != 1)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(P, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
+    if (N > 0) {
+        if (!dY || !Z) return VELORA_ERR_INVALID_ARG;
+        if (lddy < O || ldz < M) return VELORA_ERR_INVALID_ARG;
+        if (!elem_aligned(dY, dy_dtype) || !elem_aligned(Z, z_dtype)) return VELORA_ERR_ALIGNMENT;
+    }
+    if (!ws || ws_bytes < factored_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* status = static_cast<int*>(ws);
+    char* body = static_cast<char*>(ws) + kStatusBytes;
+    rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, nullptr, D, Dsub, nullptr, VELORA_F32, D, beta,
+                               body, ws_bytes - kStatusBytes, status, st, P, ldp);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    if (N == 0 && beta) return VELORA_OK;
+    return launch_gemm_simt(dY, dy_dtype, 1, lddy, Z, z_dtype, 1, ldz, P, VELORA_F32, ldp, beta, O, M, N, st);
+}
+
+int velora_expand_p(const float* P, int64_t ldp, const float* v, int64_t O, int64_t D, int Dsub,
+                    void* dW, int dw_dtype, int64_t lddw, int beta, void* stream)
+{
+    if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
+    int rc = check_shape(0, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!P || !v || !dW) return VELORA_ERR_INVALID_ARG;
+    if (!valid_dtype(dw_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (ldp < num_subtokens(D, Dsub) || lddw < D || (beta != 0 && beta != 1)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(P, VELORA_F32) || !elem_aligned(v, VELORA_F32) || !elem_aligned(dW, dw_dtype))
+        return VELORA_ERR_ALIGNMENT;
+    return launch_expand_p(P, 1, 0, ldp, v, O, D, Dsub, dW, dw_dtype, lddw, beta, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

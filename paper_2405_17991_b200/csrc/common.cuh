@@ -30,8 +30,11 @@ inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : 4; }
 inline bool valid_dtype(int dt) { return dt == VELORA_F32 || dt == VELORA_BF16; }
 
 // ---- streaming kernels (stream_kernels.cu) ----
+// sum_only != 0: v receives the un-normalised sub-token sum s and nothing is synchronised.
 int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
-                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
+                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream, int sum_only = 0);
+// v = s / ||s|| (fp64 inside), degenerate flag read back (synchronises).
+int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t init_v_workspace_bytes(int Dsub);
 int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
                     const float* v, void* Z, int z_dtype, int64_t ldz, cudaStream_t stream);

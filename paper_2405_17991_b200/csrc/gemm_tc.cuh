@@ -47,9 +47,11 @@ int read_and_clear_stream_error(cudaStream_t stream);
 
 // Factored weight gradient: P = dY^T Z on tensor cores (split over tokens), dW = P (x) v.
 size_t weight_grad_tc_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub);
+// With P_out != NULL only the factor is produced: P_out[O, M] = beta * P_out + dY^T Z (fp32), dW untouched.
 int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
                           const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
                           void* dW, int dw_dtype, int64_t lddw, int beta,
-                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream);
+                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream,
+                          float* P_out = nullptr, int64_t ldp_out = 0);
 
 }  // namespace velora

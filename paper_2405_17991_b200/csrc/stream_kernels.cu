@@ -258,7 +258,7 @@ init_v_partial_elem_kernel(const XT* __restrict__ X, int64_t N, int D, int64_t l
 // groups (independent loads), then one thread per position adds the groups in order.
 __global__ void __launch_bounds__(kStreamThreads)
 init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int Dsub,
-                       float* __restrict__ v, int* __restrict__ status)
+                       float* __restrict__ v, int* __restrict__ status, int normalize)
 {
     __shared__ double s_sum[VELORA_MAX_DSUB];
     __shared__ double s_red[kStreamThreads];
@@ -280,6 +280,10 @@ init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int
             s_sum[j] = t;
         }
         __syncthreads();
+    }
+    if (!normalize) {                                          // the plain sub-token sum s (multi-rank use)
+        for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) v[j] = static_cast<float>(s_sum[j]);
+        return;
     }
     double sq = 0.0;
     for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) sq += s_sum[j] * s_sum[j];
@@ -435,8 +439,29 @@ size_t init_v_workspace_bytes(int Dsub)
     return kStatusBytes + static_cast<size_t>(kInitVMaxCtas) * static_cast<size_t>(Dsub) * sizeof(float);
 }
 
+namespace {
+int read_degenerate_flag(const int* status, cudaStream_t stream)
+{
+    int host_status = -1;
+    if (cudaMemcpyAsync(&host_status, status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return VELORA_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (host_status == 0) return VELORA_OK;
+    return host_status == 1 ? VELORA_ERR_DEGENERATE_V : VELORA_ERR_CUDA;
+}
+}  // namespace
+
+int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    int* status = static_cast<int*>(ws) + 1;
+    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(s, 1, Dsub, v, status, 1);
+    if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+    return read_degenerate_flag(status, stream);
+}
+
 int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
-                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream)
+                  float* v, void* ws, size_t ws_bytes, cudaStream_t stream, int sum_only)
 {
     if (ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
     int* status = static_cast<int*>(ws) + 1;             // word 1: degenerate-sum flag of this call
@@ -488,15 +513,10 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
                 static_cast<const float*>(X), N, static_cast<int>(D), ldx, Dsub, M, rows_per_cta, partials);
     }
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
-    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(partials, num_partials, Dsub, v, status);
+    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(partials, num_partials, Dsub, v, status, sum_only ? 0 : 1);
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
-
-    int host_status = -1;
-    if (cudaMemcpyAsync(&host_status, status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-        return VELORA_ERR_CUDA;
-    if (cudaStreamSynchronize(stream) != cudaSuccess) return VELORA_ERR_CUDA;
-    if (host_status == 0) return VELORA_OK;
-    return host_status == 1 ? VELORA_ERR_DEGENERATE_V : VELORA_ERR_CUDA;
+    if (sum_only) return VELORA_OK;                            // v holds s; nothing to report, no synchronisation
+    return read_degenerate_flag(status, stream);
 }
 
 int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,

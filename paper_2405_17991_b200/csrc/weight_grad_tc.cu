@@ -307,6 +307,22 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
     }
 }
 
+// P[o, m] = beta * P[o, m] + sum_s partials[s][o][m], splits added in a fixed order.
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const float* __restrict__ partials, int splits, int64_t split_stride, int ldpart,
+                       int O, int M, float* __restrict__ P, int64_t ldp, int beta)
+{
+    const int64_t total = static_cast<int64_t>(O) * M;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
+        const int o = static_cast<int>(idx / M);
+        const int m = static_cast<int>(idx - static_cast<int64_t>(o) * M);
+        float p = beta ? P[o * ldp + m] : 0.f;
+        for (int s = 0; s < splits; ++s) p += __ldg(partials + s * split_stride + static_cast<int64_t>(o) * ldpart + m);
+        P[o * ldp + m] = p;
+    }
+}
+
 struct WgPlan {
     bool ok;
     int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o;
@@ -389,7 +405,8 @@ size_t weight_grad_tc_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
 int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
                           const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
                           void* dW, int dw_dtype, int64_t lddw, int beta,
-                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream)
+                          void* ws, size_t ws_bytes, int* status, cudaStream_t stream,
+                          float* P_out, int64_t ldp_out)
 {
     if (dy_dtype != VELORA_BF16 || N < 1) return VELORA_ERR_UNSUPPORTED;
     if (!tc_operand_ok(dY, lddy)) return VELORA_ERR_UNSUPPORTED;
@@ -445,6 +462,18 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
     a.beta = beta;
     a.splits = p.splits;
 
+    if (P_out) {
+        // The factor alone: P = beta * P + dY^T Z (kept across micro-batches, expanded once by the caller).
+        rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, p, di.smem_optin, stream);
+        if (rc != VELORA_OK) return rc;
+        const int64_t total = O * p.M;
+        int64_t grid = ceil_div64(total, 256);
+        const int64_t cap = static_cast<int64_t>(di.sm_count) * 8;
+        if (grid > cap) grid = cap;
+        reduce_partials_kernel<<<static_cast<int>(grid), 256, 0, stream>>>(
+            partials, p.splits, a.split_stride, p.npad, static_cast<int>(O), p.M, P_out, ldp_out, beta);
+        return after_launch();
+    }
     // 2a. one launch: cluster of the tile's splits, reduction through distributed shared memory
     const int L = (Dsub % 8 == 0) ? Dsub / 8 : 0;
     const bool vec = L >= 1 && L <= 128 && (L & (L - 1)) == 0 && aligned16(dW) &&

@@ -297,6 +297,48 @@ def test_linear_forward_backward_configs(vl, c, li, Dsub):
     assert rel_err(to_f64(dW_ex), to_f64(dW)) < TOL_GEMM
 
 
+# ------------------------------------------------------------------ factored form kept factored; sharded batches
+@pytest.mark.parametrize("c,li,Dsub", [(2, 6, 64), (3, 0, 32), (4, 0, 128), (5, 0, 64)])
+def test_factor_p_accumulates_over_micro_batches_and_expands_once(vl, c, li, Dsub):
+    cfg = vi.CONFIGS[c]
+    Xa, dYa = vi.make_X(cfg, li), vi.make_dY(cfg, li)
+    N, D = Xa.shape
+    O = dYa.shape[1]
+    ldO = -(-O // 8) * 8
+    X, dY = Xa.torch(DEV, ld=-(-D // 8) * 8), dYa.torch(DEV, ld=ldO)
+    v = vl.velora_init_v(X, Dsub)
+    v64 = to_f64(v)
+    Z = vl.velora_compress(X, v)
+    Z64, dY64 = to_f64(Z), dYa.f64()
+    cut = (N // 3 // 64) * 64 + 17                       # two uneven micro-batches
+    P = vl.velora_weight_grad_p(dY[:cut], Z[:cut], D, Dsub)
+    vl.velora_weight_grad_p(dY[cut:], Z[cut:], D, Dsub, P=P, beta=1)
+    sel = vi.sample_rows(cfg, li, O, 256, salt=3)
+    _, P_ref = oracle.weight_grad(np.ascontiguousarray(dY64[:, sel]), Z64, v64, D, factored=True, return_P=True)
+    assert_matches(P[sel], P_ref, TOL_GEMM, "P over two micro-batches")
+    dW = vl.velora_expand_p(P, v, D)
+    dW_one = vl.velora_weight_grad(dY, Z, v, D)
+    assert rel_err(to_f64(dW), to_f64(dW_one)) < TOL_GEMM
+    dW_ref = oracle.weight_grad(np.ascontiguousarray(dY64[:, sel]), Z64, v64, D, factored=True)
+    assert_matches(dW[sel], dW_ref, TOL_GEMM, "dW expanded from P")
+
+
+def test_token_sharded_init_v_gives_every_shard_the_same_v(vl):
+    cfg = vi.CONFIGS[2]
+    Xa = vi.make_X(cfg, 6)
+    X = Xa.torch(DEV)
+    N = X.shape[0]
+    shards = [X[: N // 3], X[N // 3: N // 3 + 5], X[N // 3 + 5:], X[:0]]      # uneven, one empty
+    s = sum(vl.velora_subtoken_sum(x, 64) for x in shards)                     # what the all-reduce computes
+    v = vl.velora_normalize_v(s)
+    v_ref, s_ref, _ = oracle.init_v(Xa.f64(), 64, return_sum=True)
+    assert rel_err(to_f64(s), s_ref) < 1e-4
+    assert rel_err(to_f64(v), v_ref) < 1e-4
+    assert rel_err(to_f64(v), to_f64(vl.velora_init_v(X, 64))) < 1e-5
+    with pytest.raises(vl.VeloraError):
+        vl.velora_normalize_v(torch.zeros(64, device=DEV))
+
+
 def test_chained_path_against_chained_oracle(vl):
     """init_v -> compress -> weight_grad on the GPU against the same chain in fp64 (bf16 Z storage)."""
     cfg = vi.CONFIGS[3]

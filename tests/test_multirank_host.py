@@ -64,3 +64,48 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import oracle
+    import velora_inputs as vi
+    from paper_2405_17991_b200.distributed import allreduce_sum_
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        N, D, O, Dsub = 96, 80, 12, 16
+        case = vi.small_case(77, N, D, O, dtype="bf16", mean_offset=0.2)
+        X, dY = case["X"].f64(), case["dY"].f64()
+        lo, hi = (0, 37) if rank == 0 else (37, N)            # uneven shards of the token dimension
+        # the stand-in for this rank's kernels is the oracle: what is tested is the exchange
+        _, s_local, _ = oracle.init_v(X[lo:hi], Dsub, return_sum=True)
+        s = allreduce_sum_(torch.from_numpy(s_local.copy()))
+        v = s.numpy() / np.linalg.norm(s.numpy())
+        Z_local = oracle.compress(X[lo:hi], v)
+        _, P_local = oracle.weight_grad(dY[lo:hi], Z_local, v, D, factored=True, return_P=True)
+        P = allreduce_sum_(torch.from_numpy(P_local.copy())).numpy()
+        dW = np.einsum("om,j->omj", P, v).reshape(O, -1)[:, :D]
+        v_full = oracle.init_v(X, Dsub)
+        dW_full = oracle.weight_grad(dY, oracle.compress(X, v_full), v_full, D)
+        out.put((rank, float(np.abs(v - v_full).max()), float(np.abs(dW - dW_full).max() / np.abs(dW_full).max())))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sharded_batches_reproduce_the_single_process_result():
+    """Two ranks, each with its rows: all-reducing s (Dsub floats) and P (O*M floats) gives every rank the
+    v and the dW of the undivided batch."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for _, dv, dw in results:
+        assert dv < 1e-12 and dw < 1e-12
