@@ -9,6 +9,10 @@
 // K-major (rows contiguous along K) or MN-major (rows contiguous along M or N): the latter is loaded
 // as 64 x 64 boxes and consumed through an MN-major matrix descriptor, so no transpose pass exists.
 // Ragged edges rely on TMA zero fill for loads and on predicated stores.
+#include <cstdlib>
+
+#include "gemm_fuse.cuh"
+#include "gemm_store.cuh"
 #include "gemm_tc.cuh"
 #include "tc_common.cuh"
 
@@ -28,14 +32,6 @@ constexpr int FUSE_THREADS = GEMM_THREADS + 128;    // + four compress warps
 constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256;
 constexpr size_t FUSE_SMEM = GEMM_SMEM + A_BYTES + VELORA_MAX_DSUB * 4;   // + compress tile + copy of v
 
-// Arguments of the compress that rides on the forward GEMM's A tiles (Section 3.1, Eq. 1).
-struct FuseArgs {
-    const float* v;
-    void* Z;
-    int64_t ldz;
-    int Dsub, M;
-};
-
 struct TileCoord {
     int m0, n0;
 };
@@ -52,70 +48,6 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
     const int tm = band * BAND + (in_band - tn * band_rows);
     return {tm * BM, tn * BN};
 }
-
-template <typename CT> struct Store32;
-template <> struct Store32<__nv_bfloat16> {
-    // 32 consecutive outputs of one row.
-    static __device__ __forceinline__ void run(__nv_bfloat16* p, const uint32_t (&r)[32], int valid, int beta)
-    {
-        if (valid >= 32) {
-            uint4* q = reinterpret_cast<uint4*>(p);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float f[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * i + e]);
-                if (beta) {
-                    const uint4 old = q[i];
-                    f[0] += bf16_lo(old.x); f[1] += bf16_hi(old.x);
-                    f[2] += bf16_lo(old.y); f[3] += bf16_hi(old.y);
-                    f[4] += bf16_lo(old.z); f[5] += bf16_hi(old.z);
-                    f[6] += bf16_lo(old.w); f[7] += bf16_hi(old.w);
-                }
-                uint4 o;
-                o.x = pack_bf16x2(f[0], f[1]);
-                o.y = pack_bf16x2(f[2], f[3]);
-                o.z = pack_bf16x2(f[4], f[5]);
-                o.w = pack_bf16x2(f[6], f[7]);
-                q[i] = o;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-                if (e < valid) {
-                    float f = __uint_as_float(r[e]);
-                    if (beta) f += __bfloat162float(p[e]);
-                    p[e] = __float2bfloat16_rn(f);
-                }
-        }
-    }
-};
-template <> struct Store32<float> {
-    static __device__ __forceinline__ void run(float* p, const uint32_t (&r)[32], int valid, int beta)
-    {
-        if (valid >= 32) {
-            float4* q = reinterpret_cast<float4*>(p);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float4 o = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
-                                       __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-                if (beta) {
-                    const float4 old = q[i];
-                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                }
-                q[i] = o;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-                if (e < valid) {
-                    float f = __uint_as_float(r[e]);
-                    if (beta) f += p[e];
-                    p[e] = f;
-                }
-        }
-    }
-};
 
 // FUSE = 0: plain GEMM.  FUSE = 1 / 2 (forward only, A = X K-major): Z = compress(X, v) (fp32 / bf16
 // storage) is computed by four extra warps from X tiles that are already on their way through L2 for the
@@ -269,9 +201,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (FUSE && warp >= 6) {
         // ------------------------------------------------ compress (4 warps, one tile row per thread)
         const int trow = (warp - 6) * 32 + lane;
-        const int Dsub = fz.Dsub;
-        const int nsub = Dsub >= BK ? 1 : BK / Dsub;           // sub-tokens per k-block
-        const uint32_t rowaddr = cbuf + trow * 128;
         float acc = 0.f;
         uint32_t oc = 0;
         for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
@@ -282,37 +211,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if ((kb / cw) % tiles_n != tn) continue;
                 if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
                 ++oc;
-                uint4 d[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t a = rowaddr + (static_cast<uint32_t>(c ^ (trow & 7)) << 4);
-                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(d[c].x), "=r"(d[c].y), "=r"(d[c].z), "=r"(d[c].w) : "r"(a));
-                }
-                const int j0 = (kb % cw) * BK;                 // position of this k-block inside the sub-token
-                if (kb % cw == 0) acc = 0.f;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int jv = (j0 + c * 8) & (Dsub - 1);  // Dsub is a power of two here
-                    const float4 va = *reinterpret_cast<const float4*>(sv + jv);
-                    const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
-                    if (nsub > 1 && jv == 0) acc = 0.f;        // a new sub-token starts inside the k-block
-                    float a0 = bf16_lo(d[c].x) * va.x, a1 = bf16_hi(d[c].x) * va.y;
-                    a0 = fmaf(bf16_lo(d[c].y), va.z, a0); a1 = fmaf(bf16_hi(d[c].y), va.w, a1);
-                    a0 = fmaf(bf16_lo(d[c].z), vb.x, a0); a1 = fmaf(bf16_hi(d[c].z), vb.y, a1);
-                    a0 = fmaf(bf16_lo(d[c].w), vb.z, a0); a1 = fmaf(bf16_hi(d[c].w), vb.w, a1);
-                    acc += a0 + a1;
-                    // The sub-token ends with this chunk, or the row does (ragged last sub-token: the
-                    // columns beyond D were zero-filled by TMA and no further k-block follows).
-                    if (jv + 8 == Dsub || (kb == kblocks - 1 && c == 7)) {
-                        const int m = (kb * BK + c * 8) / Dsub;
-                        if (row < Mdim && m < fz.M) {
-                            if (FUSE == 1) static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = acc;
-                            else static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
-                        }
-                    }
-                }
-                __syncwarp();                                  // every lane's reads of the tile are done
+                compress_kblock<FUSE == 2>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
+                __syncwarp();                                 // every lane's reads of the tile are done
                 if (lane == 0) mbar_arrive(cempty);
             }
         }
@@ -419,6 +319,16 @@ int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t
     return r == CUDA_SUCCESS ? VELORA_OK : VELORA_ERR_CUDA;
 }
 
+bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim)
+{
+    static const int forced = [] { const char* e = getenv("VELORA_GEMM_PAIR"); return e ? (e[0] == '1' ? 1 : 0) : -1; }();
+    if (forced >= 0) return forced == 1;
+    DeviceInfo di;
+    if (device_info(&di) != VELORA_OK) return false;
+    const int64_t pair_tiles = ((Mdim + 255) / 256) * ((Ndim + 255) / 256);
+    return pair_tiles >= di.sm_count / 2;
+}
+
 bool tc_operand_ok(const void* p, int64_t ld_elems)
 {
     return aligned16(p) && ld_elems % 8 == 0 && ld_elems * 2 < (static_cast<int64_t>(1) << 40);
@@ -435,6 +345,10 @@ int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t 
     if (!aligned16(C) || (ldc * static_cast<int64_t>(dtype_size(c_dtype))) % 16) return VELORA_ERR_UNSUPPORTED;
     if ((static_cast<int64_t>((Mdim + BM - 1) / BM) * ((Ndim + BN - 1) / BN)) > (1 << 30)) return VELORA_ERR_UNSUPPORTED;
 
+    if (gemm_pair_preferred(Mdim, Ndim)) {
+        const int prc = launch_gemm_tc_pair(kind, A, lda, B, ldb, C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, in_dtype, status, stream);
+        if (prc != VELORA_ERR_UNSUPPORTED) return prc;
+    }
     const bool a_mn = (kind == GEMM_TN_MN_MN);
     const bool b_mn = (kind != GEMM_NT_K_K);
     CUtensorMap ta, tb;
@@ -469,6 +383,10 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
     // hold the producer back, so narrow outputs take the two-kernel route as well.
     const bool wide = (O + BN - 1) / BN >= 4;
     if (pow2 && gemm_ok && wide) {
+        if (gemm_pair_preferred(N, O)) {
+            const int prc = launch_linear_forward_tc_pair(X, ldx, W, ldw, v, Y, ldy, Z, z_dtype, ldz, N, D, O, Dsub, status, stream);
+            if (prc != VELORA_ERR_UNSUPPORTED) return prc;
+        }
         CUtensorMap ta, tb;
         int rc = make_tmap_bf16_2d(&ta, X, D, N, ldx, BK, BM);
         if (rc != VELORA_OK) return rc;

@@ -22,6 +22,17 @@ int launch_gemm_tc(int kind, const void* A, int64_t lda, const void* B, int64_t 
                    void* C, int c_dtype, int64_t ldc, int beta,
                    int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream);
 
+// The same product with CTA pairs (tcgen05 cta_group::2, 256 x 256 tile per pair).  (gemm_tc2.cu)
+int launch_gemm_tc_pair(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
+                        void* C, int c_dtype, int64_t ldc, int beta,
+                        int64_t Mdim, int64_t Ndim, int64_t Kdim, int in_dtype, int* status, cudaStream_t stream);
+
+int launch_linear_forward_tc_pair(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
+                                  void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
+                                  int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
+// True when a product with this output shape fills the device with 256 x 256 pair tiles.
+bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim);
+
 // Tensor map of a row-major bf16 matrix: `inner` contiguous elements per row, `outer` rows, row pitch
 // ld_elems; 128-byte swizzle (or none), zero fill outside the matrix.  (gemm_tc.cu)
 int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
