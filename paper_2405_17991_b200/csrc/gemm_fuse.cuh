@@ -13,6 +13,20 @@ struct FuseArgs {
     int Dsub, M;
 };
 
+// Which k-blocks are compressed during the work on n-tile tn?  Those of the sub-token groups g = kb / cw
+// (cw = k-blocks per sub-token, a power of two) with g % tiles_n == tn, so that the tiles of one row block
+// share the work.  Walked incrementally: the TMA producer is a single thread on the kernel's critical
+// path, where two integer divisions per k-block cost 10 % of the run time.
+struct OwnedWalk {
+    int cwmask, tiles_n, tn, gm;
+    __device__ __forceinline__ OwnedWalk(int cw, int tiles_n_, int tn_) : cwmask(cw - 1), tiles_n(tiles_n_), tn(tn_), gm(0) {}
+    __device__ __forceinline__ bool owned() const { return gm == tn; }
+    __device__ __forceinline__ void step(int kb_next)          // call when moving on to k-block kb_next
+    {
+        if ((kb_next & cwmask) == 0 && ++gm == tiles_n) gm = 0;
+    }
+};
+
 // One thread, one row of a 128-row x 64-column bf16 X tile that TMA wrote with the 128-byte swizzle at
 // `tile` (shared-memory address, 1024-byte aligned).  Adds the row's 64 columns of k-block `kb` into the
 // running inner product `acc` with v (copy in shared memory `sv`, Dsub a power of two >= 8) and stores

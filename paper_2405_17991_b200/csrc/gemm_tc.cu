@@ -9,8 +9,6 @@
 // K-major (rows contiguous along K) or MN-major (rows contiguous along M or N): the latter is loaded
 // as 64 x 64 boxes and consumed through an MN-major matrix descriptor, so no transpose pass exists.
 // Ragged edges rely on TMA zero fill for loads and on predicated stores.
-#include <cstdlib>
-
 #include "gemm_fuse.cuh"
 #include "gemm_store.cuh"
 #include "gemm_tc.cuh"
@@ -122,7 +120,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t it = 0, oc = 0;
             for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
                 const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                OwnedWalk own(cw, tiles_n, tc0.n0 / BN);
+                for (int kb = 0; kb < kblocks; ++kb, ++it, own.step(kb)) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
                     mbar_arrive_expect_tx(full + 8 * s, A_BYTES + B_BYTES);
@@ -141,7 +140,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         tma_load_2d(sB + s * B_BYTES, &tmB, full + 8 * s, k0, tc0.n0);
                     }
-                    if (FUSE && (kb / cw) % tiles_n == tc0.n0 / BN) {      // this CTA compresses the k-block
+                    if (FUSE && own.owned()) {                             // this CTA compresses the k-block
                         if (!mbar_wait(cempty, (oc & 1u) ^ 1u, abort_flag)) { failed = true; break; }
                         mbar_arrive_expect_tx(cfull, A_BYTES);
                         tma_load_2d(cbuf, &tmA, cfull, k0, tc0.m0);
@@ -207,8 +206,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
             const int tn = tc0.n0 / BN;
             const int row = tc0.m0 + trow;
-            for (int kb = 0; kb < kblocks; ++kb) {
-                if ((kb / cw) % tiles_n != tn) continue;
+            OwnedWalk own(cw, tiles_n, tn);
+            for (int kb = 0; kb < kblocks; ++kb, own.step(kb)) {
+                if (!own.owned()) continue;
                 if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
                 ++oc;
                 compress_kblock<FUSE == 2>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
@@ -321,8 +321,6 @@ int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t
 
 bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim)
 {
-    static const int forced = [] { const char* e = getenv("VELORA_GEMM_PAIR"); return e ? (e[0] == '1' ? 1 : 0) : -1; }();
-    if (forced >= 0) return forced == 1;
     DeviceInfo di;
     if (device_info(&di) != VELORA_OK) return false;
     const int64_t pair_tiles = ((Mdim + 255) / 256) * ((Ndim + 255) / 256);

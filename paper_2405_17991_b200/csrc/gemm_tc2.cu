@@ -183,7 +183,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
                 const int m0 = t0.m0 + static_cast<int>(rank) * P_BM;
                 const int n0 = t0.n0 + static_cast<int>(rank) * (P_BN / 2);
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                OwnedWalk own(cw, tiles_n, t0.n0 / P_BN);
+                for (int kb = 0; kb < kblocks; ++kb, ++it, own.step(kb)) {
                     const uint32_t s = it % P_STAGES, ph = (it / P_STAGES) & 1u;
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
                     const uint32_t lead_full = map_to_cta(full + 8 * s, 0);
@@ -204,7 +205,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     } else {
                         tma_load_2d_pair(b_dst, &tmB, lead_full, k0, n0);
                     }
-                    if (FUSE && (kb / cw) % tiles_n == t0.n0 / P_BN) {     // this pair compresses the k-block
+                    if (FUSE && own.owned()) {                     // this pair compresses the k-block
                         if (!mbar_wait(cempty, (oc & 1u) ^ 1u, abort_flag)) { failed = true; break; }
                         mbar_arrive_expect_tx(cfull, P_A_BYTES);
                         tma_load_2d(cbuf, &tmA, cfull, k0, m0);
@@ -272,8 +273,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
             const int tn = t0.n0 / P_BN;
             const int row = t0.m0 + static_cast<int>(rank) * P_BM + trow;
-            for (int kb = 0; kb < kblocks; ++kb) {
-                if ((kb / cw) % tiles_n != tn) continue;
+            OwnedWalk own(cw, tiles_n, tn);
+            for (int kb = 0; kb < kblocks; ++kb, own.step(kb)) {
+                if (!own.owned()) continue;
                 if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
                 ++oc;
                 compress_kblock<FUSE == 2>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
