@@ -30,7 +30,7 @@ UNIT = "tokens/s"
 CONFIG_INDEX = 5
 DSUB = 64
 CPU_SAMPLE_TOKENS = 4
-GEMM_TRAFFIC_RATIO = 0.997      # ncu dram bytes / algorithmic bytes of gemm_tc_kernel on the q layer
+GEMM_TRAFFIC_RATIO = 0.985      # ncu dram bytes / algorithmic bytes of the fused forward gemm_pair_kernel on the q layer
 
 
 def peaks():
@@ -276,10 +276,11 @@ def run_ours(args):
     fwd_flops = sum(layer_flops(N, l["D"], l["O"], l["M"])["fwd"] for (l, _, _, _) in events)
     achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
     peak = pk["bf16_tflops_sustained"]
-    # DRAM traffic per launch: ncu on the q-layer launch of this kernel read + wrote 0.997 of the algorithmic
-    # bytes (every operand crosses HBM once; profiles/gemm_tc_kernel_q_layer_8192x4096x4096.md); the other
-    # layers of the step are scaled by their algorithmic bytes.
-    fwd_bytes = sum((N * l["D"] + l["O"] * l["D"] + N * l["O"]) * 2 for (l, _, _, _) in events)
+    # DRAM traffic per launch: ncu on the q-layer launch of this kernel (compress riding along) read + wrote
+    # 167.3 MB = 0.985 of the 169.9 MB of algorithmic bytes X + W + Y + Z (every operand crosses HBM once;
+    # profiles/gemm_pair_kernel_q_layer_8192x4096x4096.md); the other layers of the step run the same
+    # kernel with the same tile walk and are scaled by their algorithmic bytes.
+    fwd_bytes = sum((N * l["D"] + l["O"] * l["D"] + N * l["O"]) * 2 + N * l["M"] * 4 for (l, _, _, _) in events)
     traffic = GEMM_TRAFFIC_RATIO * fwd_bytes / max(len(events), 1)
     roofline = {"kernel": "velora_linear_forward (tensor-core GEMM Y = X W^T with compress)", "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
