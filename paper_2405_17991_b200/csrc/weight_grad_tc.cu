@@ -108,12 +108,14 @@ template <> struct WgOut8<float> {
     }
 };
 
-__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank)
+// Four consecutive floats at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t local_addr, uint32_t rank)
 {
     uint32_t remote;
-    float x;
+    float4 x;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x) : "r"(remote) : "memory");
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(remote) : "memory");
     return x;
 }
 
@@ -266,15 +268,36 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
         const int r_begin = split * rows_per;
         const int r_end = (r_begin + rows_per < WG_BM) ? r_begin + rows_per : WG_BM;
         WT* dW = static_cast<WT*>(a.dW);
+
+        // Sum the partials of this CTA's rows, all threads at once and all loads of an element in flight
+        // together (a remote load takes a good part of a microsecond; issued one after the other they
+        // outlast the whole dY stream).  The sum replaces this CTA's own partial of those rows, which no
+        // other CTA reads.
+        float* sp = reinterpret_cast<float*>(smem);
+        if (a.splits > 1) {
+            const int c4n = a.npad / 4;
+            for (int idx = threadIdx.x; idx < (r_end - r_begin) * c4n; idx += WG_THREADS) {
+                const int r = idx / c4n, c4 = idx - r * c4n;
+                const int off = (r_begin + r) * ldsp + c4 * 4;
+                const uint32_t laddr = base + static_cast<uint32_t>(off * 4);
+                float4 x[WG_MAX_SPLITS];
+#pragma unroll
+                for (int s = 0; s < WG_MAX_SPLITS; ++s)
+                    x[s] = (s < a.splits) ? ld_cluster_f32x4(laddr, static_cast<uint32_t>(s)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 t = x[0];
+#pragma unroll
+                for (int s = 1; s < WG_MAX_SPLITS; ++s) {          // fixed order
+                    t.x += x[s].x; t.y += x[s].y; t.z += x[s].z; t.w += x[s].w;
+                }
+                *reinterpret_cast<float4*>(sp + off) = t;
+            }
+            __syncthreads();
+        }
         for (int trow = r_begin + warp; trow < r_end; trow += WG_THREADS / 32) {
             const int o = o0 + trow;
             if (o >= a.O) break;
             for (int m0 = 0; m0 < a.M; m0 += 32) {
-                float p = 0.f;
-                if (m0 + lane < a.M) {
-                    const uint32_t laddr = base + static_cast<uint32_t>((trow * ldsp + m0 + lane) * 4);
-                    for (int s = 0; s < a.splits; ++s) p += ld_cluster_f32(laddr, static_cast<uint32_t>(s));   // fixed order
-                }
+                const float p = (m0 + lane < a.M) ? sp[trow * ldsp + m0 + lane] : 0.f;
                 WT* ptr = dW + static_cast<int64_t>(o) * a.lddw + (static_cast<int64_t>(m0 + sub) * L + q) * 8;
 #pragma unroll 8
                 for (int it = 0; it < LPS; ++it, ptr += SPW * L * 8) {
