@@ -44,6 +44,9 @@ template <typename ZT>
 __global__ void __launch_bounds__(256)
 z_to_bf16_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int M, int pitch, uint4* __restrict__ Zb)
 {
+    // The kernel that consumes Zb may be launched now: it waits (griddepcontrol.wait) before its first
+    // read of Zb, and meanwhile sets up and starts pulling dY.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int chunks = pitch / 8;
     const int64_t total = N * chunks;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -169,7 +172,21 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
     bool failed = false;
     if (warp == 0) {
         if (lane == 0) {
-            int it = 0;
+            // The ring starts empty: fill it with dY tiles first, then wait for the kernel that writes Zb
+            // (launched just before this one, which may overlap its tail) and add the Zb slabs.
+            const int pre = nkb < WG_STAGES ? nkb : WG_STAGES;
+            for (int it = 0; it < pre; ++it) {
+                mbar_arrive_expect_tx(full + 8 * it, static_cast<uint32_t>(stage_bytes));
+                const int k0 = (kb0 + it) * WG_BK;
+                tma_load_2d(base + it * stage_bytes, &tmY, full + 8 * it, o0, k0);
+                tma_load_2d(base + it * stage_bytes + WG_SLAB, &tmY, full + 8 * it, o0 + 64, k0);
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int it = 0; it < pre; ++it)
+                for (int i = 0; i < a.n_slabs; ++i)
+                    tma_load_2d(base + it * stage_bytes + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * it, 64 * i,
+                                (kb0 + it) * WG_BK);
+            int it = pre;
             for (; it < nkb; ++it) {
                 const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
                 if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
@@ -402,13 +419,17 @@ int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, c
     cfg.blockDim = dim3(WG_THREADS, 1, 1);
     cfg.dynamicSmemBytes = p.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = CLUSTER ? static_cast<unsigned>(p.splits) : 1u;
     attr[0].val.clusterDim.z = 1;
+    // Programmatic dependent launch: this kernel may start while the Z conversion before it in the stream
+    // is still finishing; it reads Zb only after griddepcontrol.wait.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, kern, tmY, tmZ, a) != cudaSuccess) {
         cudaGetLastError();
         return VELORA_ERR_CUDA;
