@@ -465,8 +465,10 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
     uint4* Zb = static_cast<uint4*>(ws);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + p.zb_bytes);
 
-    // 1. Z -> bf16, padded to whole 64-wide slabs
-    {
+    // 1. Z -> bf16, padded to whole 64-wide slabs.  A bf16 Z whose rows TMA can address is read in place
+    //    (columns beyond M are zero-filled by the tensor map).
+    const bool z_in_place = z_dtype == VELORA_BF16 && tc_operand_ok(Z, ldz);
+    if (!z_in_place) {
         const int64_t items = N * (p.pitch / 8);
         int64_t grid = ceil_div64(items, 256);
         const int64_t cap = static_cast<int64_t>(di.sm_count) * 8;
@@ -484,7 +486,8 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
     CUtensorMap tmY, tmZ;
     rc = make_tmap_bf16_2d(&tmY, dY, O, N, lddy, 64, WG_BK);
     if (rc != VELORA_OK) return rc;
-    rc = make_tmap_bf16_2d(&tmZ, Zb, p.pitch, N, p.pitch, 64, WG_BK);
+    rc = z_in_place ? make_tmap_bf16_2d(&tmZ, Z, p.M, N, ldz, 64, WG_BK)
+                    : make_tmap_bf16_2d(&tmZ, Zb, p.pitch, N, p.pitch, 64, WG_BK);
     if (rc != VELORA_OK) return rc;
 
     WgArgs a{};

@@ -215,6 +215,23 @@ def test_gradient_accumulation_beta_one(vl):
         assert_matches(dW, ref, TOL_GEMM, "dW accumulate")
 
 
+@pytest.mark.parametrize("N,D,O,Dsub,pad", [(1000, 3072, 776, 32, 0), (777, 1376, 520, 64, 0), (777, 1376, 520, 64, 2),
+                                            (600, 512, 264, 8, 0)])
+def test_weight_grad_takes_bf16_Z_as_stored(vl, N, D, O, Dsub, pad):
+    """bf16 Z: rows that TMA can address (pitch a multiple of 8) are read in place, others are repacked
+    first; either way the oracle gets the very Z buffer the GPU call receives."""
+    case = vi.small_case(23, N, D, O, dtype="bf16")
+    X, dY = case["X"].torch(DEV), case["dY"].torch(DEV)
+    v = vl.velora_init_v(X, Dsub)
+    M = vl.num_subtokens(D, Dsub)
+    Zbuf = torch.zeros(N, M + pad, device=DEV, dtype=torch.bfloat16)
+    Z = Zbuf[:, :M]
+    vl.velora_compress(X, v, Z=Z)
+    dW = vl.velora_weight_grad(dY, Z, v, D)
+    ref = oracle.weight_grad(case["dY"].f64(), to_f64(Z), to_f64(v), D, factored=True)
+    assert_matches(dW, ref, TOL_GEMM, "dW from bf16 Z")
+
+
 def test_empty_batch_and_degenerate_mean(vl):
     X = torch.zeros((0, 64), dtype=torch.bfloat16, device=DEV)
     v = torch.full((16,), 7.0, device=DEV)
