@@ -31,7 +31,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int WG_BM = 128, WG_BK = 64, WG_STAGES = 4;
+constexpr int WG_BM = 128, WG_BK = 64, WG_STAGES = 4;   // WG_STAGES: most ring stages (2..4 are used)
 constexpr int WG_A_BYTES = WG_BM * WG_BK * 2;         // 16 KB: two 64-wide slabs of dY^T
 constexpr int WG_SLAB = 64 * WG_BK * 2;               // 8 KB
 constexpr int WG_THREADS = 192;
@@ -69,6 +69,8 @@ struct WgArgs {
     float* partials;          // CLUSTER = false: [S][O][ldp]
     int64_t split_stride;
     int O, n_slabs, npad, tmem_cols, kblocks, kb_per_split, ldp;
+    int stages;               // ring depth, 2..WG_STAGES: as deep as still lets two CTAs share an SM
+    int tail_off;             // barriers etc. sit this far into the aligned shared memory (past ring and partial)
     int* status;
     // CLUSTER = true: the expansion
     const float* v;
@@ -132,8 +134,8 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     const int stage_bytes = WG_A_BYTES + a.n_slabs * WG_SLAB;
-    uint8_t* tail = smem + WG_STAGES * stage_bytes;
-    const uint32_t bars = base + WG_STAGES * stage_bytes;
+    uint8_t* tail = smem + a.tail_off;
+    const uint32_t bars = base + a.tail_off;
     const uint32_t full = bars, empty = bars + 8 * WG_STAGES, tfull = bars + 16 * WG_STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * WG_STAGES + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * WG_STAGES + 24);
@@ -174,7 +176,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
         if (lane == 0) {
             // The ring starts empty: fill it with dY tiles first, then wait for the kernel that writes Zb
             // (launched just before this one, which may overlap its tail) and add the Zb slabs.
-            const int pre = nkb < WG_STAGES ? nkb : WG_STAGES;
+            const int pre = nkb < a.stages ? nkb : a.stages;
             for (int it = 0; it < pre; ++it) {
                 mbar_arrive_expect_tx(full + 8 * it, static_cast<uint32_t>(stage_bytes));
                 const int k0 = (kb0 + it) * WG_BK;
@@ -187,8 +189,8 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
                     tma_load_2d(base + it * stage_bytes + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * it, 64 * i,
                                 (kb0 + it) * WG_BK);
             int it = pre;
+            uint32_t s = 0, ph = 1;                          // stage and phase parity of iteration `it` (= stages here)
             for (; it < nkb; ++it) {
-                const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
                 if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
                 mbar_arrive_expect_tx(full + 8 * s, static_cast<uint32_t>(stage_bytes));
                 const int k0 = (kb0 + it) * WG_BK;
@@ -197,14 +199,15 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
                 tma_load_2d(a_dst + WG_SLAB, &tmY, full + 8 * s, o0 + 64, k0);
                 for (int i = 0; i < a.n_slabs; ++i)
                     tma_load_2d(a_dst + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * s, 64 * i, k0);
+                if (++s == static_cast<uint32_t>(a.stages)) { s = 0; ph ^= 1u; }
             }
             if (failed) {
                 *abort_flag = 1;
-                const int back = it < WG_STAGES ? it : WG_STAGES;   // copies of this CTA still in flight
+                const int back = it < a.stages ? it : a.stages;   // copies of this CTA still in flight
                 for (int j = 1; j <= back; ++j) {
                     const int jt = it - j;
                     const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full + 8 * (jt % WG_STAGES), (jt / WG_STAGES) & 1u))
+                    while (!mbar_try_wait(full + 8 * (jt % a.stages), (jt / a.stages) & 1u))
                         if (globaltimer_ns() - t0 > kWaitLimitNs) break;
                 }
             }
@@ -212,8 +215,8 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(WG_BM, a.npad, true, true);
+            uint32_t s = 0, ph = 0;
             for (int it = 0; it < nkb; ++it) {
-                const uint32_t s = it % WG_STAGES, ph = (it / WG_STAGES) & 1u;
                 if (!mbar_wait(full + 8 * s, ph, abort_flag)) { failed = true; break; }
                 tc_fence_after_sync();
                 const uint32_t a_addr = base + s * stage_bytes, b_addr = a_addr + WG_A_BYTES;
@@ -224,6 +227,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
                     umma_bf16(tmem_base, da, db, idesc, (it | j) != 0);
                 }
                 umma_commit(empty + 8 * s);
+                if (++s == static_cast<uint32_t>(a.stages)) { s = 0; ph ^= 1u; }
             }
             if (!failed) umma_commit(tfull);
             else *abort_flag = 1;
@@ -365,7 +369,7 @@ reduce_partials_kernel(const float* __restrict__ partials, int splits, int64_t s
 
 struct WgPlan {
     bool ok;
-    int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o;
+    int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o, stages, tail_off;
     size_t zb_bytes, part_bytes, smem;
 };
 
@@ -382,7 +386,20 @@ WgPlan make_plan(int64_t N, int64_t D, int64_t O, int Dsub, int sm_count)
     while (p.tmem_cols < p.npad) p.tmem_cols *= 2;
     p.kblocks = static_cast<int>(ceil_div64(N, WG_BK));
     p.tiles_o = static_cast<int>(ceil_div64(O, WG_BM));
-    p.smem = 1024 + static_cast<size_t>(WG_STAGES) * (WG_A_BYTES + p.n_slabs * WG_SLAB) + 256;
+    // Shared memory holds the ring and, afterwards, the CTA's partial product (128 rows of npad + 4 floats).
+    // The ring is as deep as still lets two CTAs share an SM (down to two stages: with two CTAs pulling,
+    // as many bytes are in flight per SM as with one CTA and four stages, and twice the warps write dW).
+    const size_t stage_bytes = WG_A_BYTES + static_cast<size_t>(p.n_slabs) * WG_SLAB;
+    const size_t partial_bytes = static_cast<size_t>(WG_BM) * (p.npad + 4) * 4;
+    auto smem_for = [&](int stages) {
+        const size_t body = stages * stage_bytes > partial_bytes ? stages * stage_bytes : partial_bytes;
+        return 1024 + ((body + 1023) / 1024) * 1024 + 256;
+    };
+    p.stages = WG_STAGES;
+    while (p.stages > 2 && 2 * (smem_for(p.stages) + 1024) > 228 * 1024) --p.stages;
+    if (2 * (smem_for(p.stages) + 1024) > 228 * 1024) p.stages = WG_STAGES;      // one CTA per SM either way
+    p.smem = smem_for(p.stages);
+    p.tail_off = static_cast<int>(p.smem - 1024 - 256);
     const int64_t slots = static_cast<int64_t>(sm_count) * (2 * (p.smem + 1024) <= 228 * 1024 ? 2 : 1);
     // Pick the split count that fills whole waves of SMs best; ties go to fewer splits (fewer partials).
     int best = 1;
@@ -499,6 +516,8 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
     a.tmem_cols = p.tmem_cols;
     a.kblocks = p.kblocks;
     a.kb_per_split = p.kb_per_split;
+    a.stages = p.stages;
+    a.tail_off = p.tail_off;
     a.ldp = p.npad;
     a.status = status;
     a.v = v;
@@ -525,7 +544,7 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
     const int L = (Dsub % 8 == 0) ? Dsub / 8 : 0;
     const bool vec = L >= 1 && L <= 128 && (L & (L - 1)) == 0 && aligned16(dW) &&
                      (lddw * static_cast<int64_t>(dtype_size(dw_dtype))) % 16 == 0 &&
-                     static_cast<size_t>(WG_BM) * (p.npad + 4) * 4 <= static_cast<size_t>(WG_STAGES) * (WG_A_BYTES + p.n_slabs * WG_SLAB);
+                     static_cast<size_t>(WG_BM) * (p.npad + 4) * 4 <= static_cast<size_t>(p.tail_off);
     if (vec) {
         const int lps = L < 32 ? L : 32, ch = L / lps;
         rc = VELORA_ERR_CUDA;
