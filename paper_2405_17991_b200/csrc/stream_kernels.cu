@@ -270,8 +270,16 @@ init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int
         const int slot = threadIdx.x / width;
         double s = 0.0;
         if (slot < slots)
-            for (int b = slot; b < num_partials; b += slots)
-                s += static_cast<double>(partials[static_cast<int64_t>(b) * Dsub + j]);
+            for (int b = slot; b < num_partials; b += 8 * slots) {     // eight loads in flight, added in order
+                float x[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int bu = b + u * slots;
+                    x[u] = bu < num_partials ? partials[static_cast<int64_t>(bu) * Dsub + j] : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) s += static_cast<double>(x[u]);
+            }
         s_red[threadIdx.x] = s;
         __syncthreads();
         if (threadIdx.x < width) {
