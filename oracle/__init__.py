@@ -51,6 +51,8 @@ def _load():
         lib.velora_oracle_threads.restype = ctypes.c_int
         lib.velora_oracle_threads.argtypes = []
         lib.velora_oracle_init_v.argtypes = [_p, _i64, _i64, _i64, _i64, _p, _p, _p]
+        lib.velora_oracle_update_v.argtypes = [_p, _i64, _i64, _i64, _i64, ctypes.c_double, _p, _p, _p]
+        lib.velora_oracle_update_v.restype = ctypes.c_int
         lib.velora_oracle_compress.argtypes = [_p, _i64, _i64, _i64, _i64, _p, _p, _i64]
         lib.velora_oracle_reconstruct.argtypes = [_p, _i64, _i64, _i64, _i64, _p, _p, _i64]
         lib.velora_oracle_weight_grad_bruteforce.argtypes = [
@@ -109,6 +111,21 @@ def init_v(X, Dsub, return_sum=False):
     if return_sum:
         return v, s, norm.value
     return v
+
+
+def update_v(X, Dsub, rho, a=None):
+    """Running-average variant (Section 5, initialisation ablation): a' = (1-rho) a + rho mean, v = a'/||a'||.
+
+    Returns (a', v)."""
+    X = _f64(X, 2)
+    N, D = X.shape
+    a_in = None if a is None else _f64(a, 1)
+    a_out = np.zeros(Dsub, dtype=np.float64)
+    v = np.zeros(Dsub, dtype=np.float64)
+    rc = _load().velora_oracle_update_v(_ptr(X), N, D, D, Dsub, float(rho),
+                                        _ptr(a_in) if a_in is not None else None, _ptr(a_out), _ptr(v))
+    _check(rc, "update_v")
+    return a_out, v
 
 
 def compress(X, v):

@@ -28,8 +28,10 @@
  * Pythagoras, exact cases (multiples of v, Dsub = 1, constant input),
  * idempotence, linearity, sign flip, sum(Z) = ||s||, brute force vs factored
  * weight gradient, the closed form dW = (dY^T X)(I (x) v v^T) against
- * numpy's matmul, and textbook GEMMs against numpy's matmul.
- * No function here is "parity unpinned".
+ * numpy's matmul, and textbook GEMMs against numpy's matmul; the running
+ * average against init_v (rho = 1; rho = 1/t over equal batches) and its
+ * fixed points.  No function here is "parity unpinned"; what the running
+ * average's formula should be is a reading of the paper, stated above it.
  */
 #include <math.h>
 #include <stddef.h>
@@ -87,6 +89,47 @@ int velora_oracle_init_v(const double *X, int64_t N, int64_t D, int64_t ldx, int
     if (norm_out) *norm_out = norm;
     if (!(norm > 0.0) || !isfinite(norm)) return ORACLE_DEGENERATE_V;
     for (int64_t j = 0; j < Dsub; ++j) v[j] = s[j] / norm;
+    return ORACLE_OK;
+}
+
+/*
+ * Running-average variant of the initialisation (Section 5, "Initialisation
+ * strategy": the "Running average" row of the ablation table).  The paper
+ * names the variant and gives no formula; the reading taken here is an
+ * exponential average of the per-batch sub-token means, re-normalised:
+ *   mean[j] = (1 / (N*M)) * sum_n sum_m Xp[n, m*Dsub + j]
+ *   a'[j]   = (1 - rho) * a[j] + rho * mean[j]          (rho == 1: a' = mean, a is not read)
+ *   v       = a' / ||a'||_2
+ * rho = 1 follows every incoming batch; rho = 1/t at the t-th batch makes a'
+ * the mean of everything seen so far (equal-size batches), whose direction is
+ * the fixed-average v of velora_oracle_init_v on the concatenated batches.
+ * Returns ORACLE_DEGENERATE_V (a_out, v untouched) if ||a'|| is zero or not finite.
+ */
+int velora_oracle_update_v(const double *X, int64_t N, int64_t D, int64_t ldx, int64_t Dsub,
+                           double rho, const double *a, double *a_out, double *v)
+{
+    if (!X || !v || !a_out || N < 1 || D < 1 || Dsub < 1 || Dsub > D || ldx < D) return ORACLE_BAD_ARG;
+    if (Dsub > 4096 || (rho != 1.0 && !a)) return ORACLE_BAD_ARG;
+    const int64_t M = count_subtokens(D, Dsub);
+    double an[4096];
+    for (int64_t j = 0; j < Dsub; ++j) {
+        double sum = 0.0;
+        for (int64_t n = 0; n < N; ++n)
+            for (int64_t m = 0; m < M; ++m) {
+                const int64_t d = m * Dsub + j;
+                if (d < D) sum += X[n * ldx + d];
+            }
+        const double mean = sum / ((double)N * (double)M);
+        an[j] = (rho == 1.0) ? mean : (1.0 - rho) * a[j] + rho * mean;
+    }
+    double sq = 0.0;
+    for (int64_t j = 0; j < Dsub; ++j) sq += an[j] * an[j];
+    const double norm = sqrt(sq);
+    if (!(norm > 0.0) || !isfinite(norm)) return ORACLE_DEGENERATE_V;
+    for (int64_t j = 0; j < Dsub; ++j) {
+        a_out[j] = an[j];
+        v[j] = an[j] / norm;
+    }
     return ORACLE_OK;
 }
 

@@ -278,6 +278,49 @@ def test_pins_detect_planted_mistakes():
     assert _rel(oracle.weight_grad(dY, Z, v, D), good) < 1e-12
 
 
+# --- running-average variant of the initialisation (Section 5, ablation on the initialisation strategy) ---
+
+def test_running_average_with_rho_one_is_the_fixed_average_of_that_batch():
+    X, _, _ = _case(31, 40, 72, 3, offset=0.3)
+    for Dsub in (8, 16, 24):                       # 16 leaves a ragged last sub-token (72 = 4 * 16 + 8)
+        a, v = oracle.update_v(X, Dsub, 1.0)
+        assert _rel(v, oracle.init_v(X, Dsub)) < 1e-12
+        Xp, M = _pad(X, Dsub)
+        assert _rel(a, Xp.reshape(-1, Dsub).mean(axis=0)) < 1e-12
+        assert abs(np.linalg.norm(v) - 1.0) < 1e-12
+
+
+def test_running_average_with_rho_one_over_t_is_the_fixed_average_of_all_batches_seen():
+    N, D, Dsub, T = 24, 64, 16, 5
+    batches = [_case(40 + t, N, D, 2, offset=0.1 * t)[0] for t in range(T)]
+    a = None
+    for t, X in enumerate(batches, start=1):
+        a, v = oracle.update_v(X, Dsub, 1.0 / t, a)
+        assert _rel(v, oracle.init_v(np.concatenate(batches[:t], axis=0), Dsub)) < 1e-12
+
+
+def test_running_average_fixed_points_and_mixing():
+    X, _, _ = _case(33, 30, 48, 2, offset=0.5)
+    Dsub = 16
+    mean, v_mean = oracle.update_v(X, Dsub, 1.0)
+    # rho = 0 keeps the state; feeding the same batch again keeps the direction for any rho
+    a0 = np.linspace(1.0, 2.0, Dsub)
+    a, v = oracle.update_v(X, Dsub, 0.0, a0)
+    assert _rel(a, a0) < 1e-15 and _rel(v, a0 / np.linalg.norm(a0)) < 1e-15
+    a, v = oracle.update_v(X, Dsub, 0.3, mean)
+    assert _rel(a, mean) < 1e-12 and _rel(v, v_mean) < 1e-12
+    # the state is the convex combination, written out with numpy
+    a, v = oracle.update_v(X, Dsub, 0.25, a0)
+    expect = 0.75 * a0 + 0.25 * X.reshape(-1, Dsub).mean(axis=0)
+    assert _rel(a, expect) < 1e-12 and _rel(v, expect / np.linalg.norm(expect)) < 1e-12
+    # a planted mistake (sum instead of mean, or the weights swapped) is seen by the pins above
+    wrong_sum = 0.75 * a0 + 0.25 * X.reshape(-1, Dsub).sum(axis=0)
+    wrong_swap = 0.25 * a0 + 0.75 * X.reshape(-1, Dsub).mean(axis=0)
+    assert _rel(wrong_sum, a) > 1e-2 and _rel(wrong_swap, a) > 1e-2
+    with pytest.raises(oracle.OracleError):
+        oracle.update_v(np.zeros((4, 32)), 16, 1.0)
+
+
 # --- value-format helpers ---
 
 def test_bf16_rounding_helper_matches_bit_level_rounding():
