@@ -72,7 +72,8 @@ typedef enum {
     VELORA_OP_WEIGHT_GRAD_EXPLICIT = 2,
     VELORA_OP_LINEAR_FORWARD = 3,
     VELORA_OP_LINEAR_BACKWARD_FACTORED = 4,
-    VELORA_OP_LINEAR_BACKWARD_EXPLICIT = 5
+    VELORA_OP_LINEAR_BACKWARD_EXPLICIT = 5,
+    VELORA_OP_UPDATE_V = 6
 } velora_op;
 
 #define VELORA_MAX_DSUB 1024
@@ -98,7 +99,8 @@ size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
  * fed by a tile copy or by the tensor cores) gives up after one second instead of spinning for ever.
  * velora_workspace_init zeroes the header (asynchronously, on `stream`): call it once after
  * allocating a workspace.  velora_workspace_status synchronises `stream`, reads the flag and returns
- * VELORA_OK or VELORA_ERR_TIMEOUT; outputs of a call that raised the flag are undefined.
+ * VELORA_OK or VELORA_ERR_TIMEOUT; outputs of a call that raised the flag are undefined.  (The one other
+ * value is VELORA_ERR_DEGENERATE_V, which velora_update_v leaves there instead of synchronising.)
  * The paper has no counterpart: this is run-time hygiene of the implementation.
  */
 int velora_workspace_init(void* ws, size_t ws_bytes, void* stream);
@@ -217,12 +219,31 @@ int velora_subtoken_sum(const void* X, int x_dtype, int64_t N, int64_t D, int64_
 int velora_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Running-average variant of the initialisation (Section 5, ablation on the initialisation strategy,
+ * row "Running average").  The paper names the variant without a formula; the reading implemented is an
+ * exponential average of the per-batch sub-token means, re-normalised:
+ *   a[j] <- (1 - rho) * a[j] + rho * s[j] / (N * M),  s as in velora_subtoken_sum;   v <- a / ||a||_2
+ * rho in [0, 1].  rho = 1 makes v follow each incoming batch (a is not read, so it needs no initial value);
+ * rho = 1/t at the t-th call of equal-size batches keeps a at the mean of everything seen, i.e. v at the
+ * fixed average of velora_init_v over the concatenated batches.
+ * a[Dsub], v[Dsub]: device fp32, the caller's running state and the vector to use from now on.
+ * Asynchronous (no synchronisation).  If ||a|| comes out zero or not finite, a and v are left as they
+ * were and the workspace's status word is set: velora_workspace_status then returns
+ * VELORA_ERR_DEGENERATE_V until velora_workspace_init.  N == 0 changes nothing.
+ * ws: velora_workspace_bytes(VELORA_OP_UPDATE_V, ...) bytes, initialised once with velora_workspace_init.
+ */
+int velora_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
+                    float* a, float* v, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * The factored weight gradient kept in factored form (the rank-1 structure of Section 3.2, per sub-token):
  *   velora_weight_grad_p:  P[O, M] = beta * P + dY^T Z      (fp32, ldp >= M)
  *   velora_expand_p:       dW[o, m*Dsub + j] = beta * dW + P[o, m] * v[j]
  * Since v is frozen, P can be accumulated over micro-batches (beta = 1) and summed over data-parallel
  * ranks (an all-reduce of O*M floats instead of O*D gradients) before it is expanded ONCE; the two calls in
  * sequence give the same dW as velora_weight_grad in VELORA_WG_FACTORED mode.
+ * Because the expansion is linear in v, a plain gradient step needs no dW at all: velora_expand_p with
+ * beta = 1, the weight matrix as `dW` and a copy of v scaled by -lr gives W <- W - lr * (P (x) v).
  * ws of velora_weight_grad_p: velora_workspace_bytes(VELORA_OP_WEIGHT_GRAD_FACTORED, N, D, O, Dsub).
  */
 int velora_weight_grad_p(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,

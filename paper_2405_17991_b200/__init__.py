@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     velora_linear_backward, velora_linear_forward, velora_reconstruct, velora_status_string,
     velora_version, velora_weight_grad, velora_workspace_alloc, velora_workspace_bytes,
     velora_workspace_init, velora_workspace_status, velora_launch_count, velora_device_error, velora_subtoken_sum, velora_normalize_v,
+    velora_update_v, OP_UPDATE_V, ERR_DEGENERATE_V,
     velora_weight_grad_p, velora_expand_p,
     velora_host_step_staging_bytes, velora_linear_step_host,
 )

@@ -21,7 +21,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_DEGENERA
 F32, BF16 = 0, 1
 WG_FACTORED, WG_EXPLICIT = 0, 1
 (OP_INIT_V, OP_WEIGHT_GRAD_FACTORED, OP_WEIGHT_GRAD_EXPLICIT, OP_LINEAR_FORWARD,
- OP_LINEAR_BACKWARD_FACTORED, OP_LINEAR_BACKWARD_EXPLICIT) = range(6)
+ OP_LINEAR_BACKWARD_FACTORED, OP_LINEAR_BACKWARD_EXPLICIT, OP_UPDATE_V) = range(7)
 
 _p, _i64, _int, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
 
@@ -39,6 +39,7 @@ SIGNATURES = {
     "velora_init_v_static": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p]),
     "velora_subtoken_sum": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
     "velora_normalize_v": (_int, [_p, _int, _p, _p, _sz, _p]),
+    "velora_update_v": (_int, [_p, _int, _i64, _i64, _i64, _int, ctypes.c_float, _p, _p, _p, _sz, _p]),
     "velora_weight_grad_p": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _i64, _int, _p, _i64, _int, _p, _sz, _p]),
     "velora_expand_p": (_int, [_p, _i64, _p, _i64, _i64, _int, _p, _int, _i64, _int, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
@@ -126,7 +127,8 @@ def velora_workspace_init(ws: torch.Tensor, stream=None) -> None:
 
 
 def velora_workspace_status(ws: torch.Tensor, stream=None) -> int:
-    """Synchronises the stream; 0 or ERR_TIMEOUT if a kernel's bounded wait expired."""
+    """Synchronises the stream; 0, ERR_TIMEOUT if a kernel's bounded wait expired, or ERR_DEGENERATE_V
+    left by velora_update_v."""
     return int(lib().velora_workspace_status(ctypes.c_void_p(ws.data_ptr()), _stream(stream)))
 
 
@@ -324,6 +326,18 @@ def velora_subtoken_sum(X: torch.Tensor, Dsub: int, s: Optional[torch.Tensor] = 
                                    _stream(stream))
     _check(rc, "velora_subtoken_sum")
     return s
+
+
+def velora_update_v(X: torch.Tensor, Dsub: int, rho: float, a: torch.Tensor, v: torch.Tensor,
+                    ws: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Running-average variant: a <- (1 - rho) a + rho * (mean sub-token of X), v <- a / ||a||, in place, no sync."""
+    xp, ldx = _mat(X, "X")
+    N, D = X.shape
+    if ws is None:
+        ws = velora_workspace_alloc(velora_workspace_bytes(OP_UPDATE_V, N, D, 1, Dsub), X.device)
+    rc = lib().velora_update_v(xp, _dt(X), N, D, ldx, Dsub, float(rho), _vec(a), _vec(v),
+                               ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_update_v")
 
 
 def velora_normalize_v(s: torch.Tensor, v: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,

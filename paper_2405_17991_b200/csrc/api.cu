@@ -147,7 +147,8 @@ int velora_workspace_status(const void* ws, void* stream)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return VELORA_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return VELORA_ERR_CUDA;
-    return word == 0 ? VELORA_OK : VELORA_ERR_TIMEOUT;
+    if (word == 0) return VELORA_OK;
+    return word == VELORA_ERR_DEGENERATE_V ? VELORA_ERR_DEGENERATE_V : VELORA_ERR_TIMEOUT;
 }
 
 const char* velora_status_string(int status)
@@ -175,6 +176,7 @@ size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
         case VELORA_OP_WEIGHT_GRAD_EXPLICIT:
         case VELORA_OP_LINEAR_BACKWARD_EXPLICIT: return xhat_bytes(N, D);
         case VELORA_OP_LINEAR_FORWARD: return kStatusBytes;
+        case VELORA_OP_UPDATE_V: return update_v_workspace_bytes(Dsub);
         default: return 0;
     }
 }
@@ -370,6 +372,22 @@ int velora_subtoken_sum(const void* X, int x_dtype, int64_t N, int64_t D, int64_
     if (!ws || ws_bytes < init_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
     if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
     return launch_init_v(X, x_dtype, N, D, ldx, Dsub, s, ws, ws_bytes, st, 1);
+}
+
+int velora_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
+                    float* a, float* v, void* ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!(rho >= 0.f && rho <= 1.f)) return VELORA_ERR_INVALID_ARG;
+    if (N == 0) return VELORA_OK;                         /* an empty batch has no mean: a and v stay */
+    if (!X || !a || !v) return VELORA_ERR_INVALID_ARG;
+    if (ldx < D) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(X, x_dtype) || !elem_aligned(a, VELORA_F32) || !elem_aligned(v, VELORA_F32)) return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < update_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return launch_update_v(X, x_dtype, N, D, ldx, Dsub, rho, a, v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 int velora_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, void* stream)

@@ -36,6 +36,9 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
 // v = s / ||s|| (fp64 inside), degenerate flag read back (synchronises).
 int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t init_v_workspace_bytes(int Dsub);
+size_t update_v_workspace_bytes(int Dsub);
+int launch_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
+                    float* a, float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
 int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
                     const float* v, void* Z, int z_dtype, int64_t ldz, cudaStream_t stream);
 int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,

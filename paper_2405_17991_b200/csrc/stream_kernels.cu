@@ -310,6 +310,44 @@ init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int
         for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) v[j] = static_cast<float>(s_sum[j] / norm);
 }
 
+// Running-average variant of the initialisation (Section 5, ablation on the initialisation strategy):
+//   a <- (1 - rho) * a + rho * s / count,   v <- a / ||a||_2      (rho == 1: a is not read)
+// s is this batch's sub-token sum.  One CTA; fp64 like init_v_finalize_kernel.  A zero or non-finite norm
+// leaves a and v as they were and raises the workspace's sticky status word.
+__global__ void __launch_bounds__(kStreamThreads)
+update_v_kernel(const float* __restrict__ s, double inv_count, float rho, int Dsub,
+                float* __restrict__ a, float* __restrict__ v, int* __restrict__ sticky)
+{
+    __shared__ double s_a[VELORA_MAX_DSUB];
+    __shared__ double s_red[kStreamThreads];
+    __shared__ double s_norm;
+    double sq = 0.0;
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) {
+        const double mean = static_cast<double>(s[j]) * inv_count;
+        const double an = (rho == 1.f) ? mean
+                                       : (1.0 - static_cast<double>(rho)) * static_cast<double>(a[j]) + static_cast<double>(rho) * mean;
+        s_a[j] = an;
+        sq += an * an;
+    }
+    s_red[threadIdx.x] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < kStreamThreads; ++i) t += s_red[i];
+        s_norm = sqrt(t);
+    }
+    __syncthreads();
+    const double norm = s_norm;
+    if (!((norm > 0.0) && isfinite(norm))) {
+        if (threadIdx.x == 0) atomicCAS(sticky, 0, VELORA_ERR_DEGENERATE_V);
+        return;
+    }
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) {
+        a[j] = static_cast<float>(s_a[j]);
+        v[j] = static_cast<float>(s_a[j] / norm);
+    }
+}
+
 // ------------------------------------------------------------------ compress / reconstruct (element-wise)
 template <typename XT, typename ZT>
 __global__ void __launch_bounds__(kStreamThreads)
@@ -466,6 +504,23 @@ int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_b
     init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(s, 1, Dsub, v, status, 1);
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
     return read_degenerate_flag(status, stream);
+}
+
+size_t update_v_workspace_bytes(int Dsub)
+{
+    return init_v_workspace_bytes(Dsub) + ((static_cast<size_t>(Dsub) * sizeof(float) + 255) / 256) * 256;
+}
+
+int launch_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
+                    float* a, float* v, void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (ws_bytes < update_v_workspace_bytes(Dsub)) return VELORA_ERR_WORKSPACE;
+    float* s = reinterpret_cast<float*>(static_cast<char*>(ws) + init_v_workspace_bytes(Dsub));
+    const int rc = launch_init_v(X, x_dtype, N, D, ldx, Dsub, s, ws, init_v_workspace_bytes(Dsub), stream, 1);
+    if (rc != VELORA_OK) return rc;
+    const double count = static_cast<double>(N) * static_cast<double>(ceil_div64(D, Dsub));
+    update_v_kernel<<<1, kStreamThreads, 0, stream>>>(s, 1.0 / count, rho, Dsub, a, v, static_cast<int*>(ws));
+    return check_launch();
 }
 
 int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,

@@ -340,6 +340,21 @@ def test_factor_p_accumulates_over_micro_batches_and_expands_once(vl, c, li, Dsu
     assert_matches(dW[sel], dW_ref, TOL_GEMM, "dW expanded from P")
 
 
+def test_gradient_step_straight_from_the_factor(vl):
+    """W <- W - lr * (P (x) v) through velora_expand_p (beta = 1, v scaled by -lr): no dW buffer."""
+    case = vi.small_case(29, 600, 512, 264, dtype="bf16")
+    X, dY = case["X"].torch(DEV), case["dY"].torch(DEV)
+    W = case["W"].torch(DEV).float()                   # fp32 master weights
+    Dsub, lr = 32, 0.125
+    v = vl.velora_init_v(X, Dsub)
+    Z = vl.velora_compress(X, v)
+    P = vl.velora_weight_grad_p(dY, Z, 512, Dsub)
+    W_ref = case["W"].f64() - lr * oracle.weight_grad(case["dY"].f64(), to_f64(Z), to_f64(v), 512, factored=True)
+    vl.velora_expand_p(P, v * (-lr), 512, dW=W, beta=1)
+    assert_matches(W, W_ref, TOL_GEMM, "W after the step")
+    assert rel_err(to_f64(W) - case["W"].f64(), W_ref - case["W"].f64()) < TOL_GEMM
+
+
 def test_token_sharded_init_v_gives_every_shard_the_same_v(vl):
     cfg = vi.CONFIGS[2]
     Xa = vi.make_X(cfg, 6)
@@ -354,6 +369,35 @@ def test_token_sharded_init_v_gives_every_shard_the_same_v(vl):
     assert rel_err(to_f64(v), to_f64(vl.velora_init_v(X, 64))) < 1e-5
     with pytest.raises(vl.VeloraError):
         vl.velora_normalize_v(torch.zeros(64, device=DEV))
+
+
+@pytest.mark.parametrize("N,D,Dsub,dtype", [(8192, 4096, 64, "bf16"), (777, 1376, 64, "bf16"), (300, 200, 24, "f32"),
+                                             (1000, 768, 32, "bf16")])
+def test_running_average_v_follows_the_oracle_over_several_batches(vl, N, D, Dsub, dtype):
+    """velora_update_v (running-average initialisation): three batches with rho = 1, 1/2, 0.3."""
+    a = torch.zeros(Dsub, device=DEV)
+    v = torch.zeros(Dsub, device=DEV)
+    ws = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_UPDATE_V, N, D, 1, Dsub), DEV)
+    a_ref = None
+    for t, rho in enumerate((1.0, 0.5, 0.3)):
+        X = vi.small_case(50 + t, N, D, 8, dtype=dtype, mean_offset=0.05 * (t + 1))["X"]
+        vl.velora_update_v(X.torch(DEV), Dsub, rho, a, v, ws=ws)
+        a_ref, v_ref = oracle.update_v(X.f64(), Dsub, rho, a_ref)
+        assert rel_err(to_f64(a), a_ref) < 1e-5
+        assert rel_err(to_f64(v), v_ref) < 1e-5
+        a_ref = to_f64(a)                              # the state the next GPU call reads is the stored fp32 one
+    assert vl.velora_workspace_status(ws) == 0
+    # rho = 1 is init_v of the batch
+    X = vi.small_case(60, N, D, 8, dtype=dtype, mean_offset=0.1)["X"].torch(DEV)
+    vl.velora_update_v(X, Dsub, 1.0, a, v, ws=ws)
+    assert rel_err(to_f64(v), to_f64(vl.velora_init_v(X, Dsub))) < 1e-5
+    # a zero batch at rho = 1 has no direction: state kept, sticky status raised, no exception, no sync
+    before = v.clone()
+    vl.velora_update_v(torch.zeros_like(X), Dsub, 1.0, a, v, ws=ws)
+    assert vl.velora_workspace_status(ws) == vl.ERR_DEGENERATE_V
+    assert torch.equal(v, before)
+    vl.velora_workspace_init(ws)
+    assert vl.velora_workspace_status(ws) == 0
 
 
 def test_chained_path_against_chained_oracle(vl):
