@@ -25,6 +25,24 @@ int device_info(DeviceInfo* out);
 int after_launch();
 
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+// Programmatic dependent launch.  A kernel launched with pdl_attribute() may become resident while the
+// kernel before it in the stream is still running; it must call pdl_wait() before it touches anything
+// that kernel writes (the wait returns once that kernel has completed and its writes are visible).
+// pdl_trigger() in a kernel lets the NEXT kernel in the stream, if launched this way, start early.
+// Used between the Z conversion and the weight-gradient kernel; tried on the dense products as well,
+// where hiding the launch latency of a 200-500 us kernel made no measurable difference.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+inline cudaLaunchAttribute pdl_attribute()
+{
+    cudaLaunchAttribute a{};
+    a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    a.val.programmaticStreamSerializationAllowed = 1;
+    return a;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : 4; }
 inline bool valid_dtype(int dt) { return dt == VELORA_F32 || dt == VELORA_BF16; }

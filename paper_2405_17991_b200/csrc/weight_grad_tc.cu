@@ -45,8 +45,9 @@ __global__ void __launch_bounds__(256)
 z_to_bf16_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int M, int pitch, uint4* __restrict__ Zb)
 {
     // The kernel that consumes Zb may be launched now: it waits (griddepcontrol.wait) before its first
-    // read of Zb, and meanwhile sets up and starts pulling dY.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // read of Zb, and meanwhile sets up and starts pulling dY.  Z itself may come from the kernel before.
+    pdl_trigger();
+    pdl_wait();
     const int chunks = pitch / 8;
     const int64_t total = N * chunks;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -183,7 +184,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
                 tma_load_2d(base + it * stage_bytes, &tmY, full + 8 * it, o0, k0);
                 tma_load_2d(base + it * stage_bytes + WG_SLAB, &tmY, full + 8 * it, o0 + 64, k0);
             }
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+            pdl_wait();
             for (int it = 0; it < pre; ++it)
                 for (int i = 0; i < a.n_slabs; ++i)
                     tma_load_2d(base + it * stage_bytes + WG_A_BYTES + i * WG_SLAB, &tmZ, full + 8 * it, 64 * i,
@@ -370,6 +371,7 @@ reduce_partials_kernel(const float* __restrict__ partials, int splits, int64_t s
 struct WgPlan {
     bool ok;
     int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o, stages, tail_off;
+    bool after_conversion;    // the launch follows z_to_bf16_kernel in the stream
     size_t zb_bytes, part_bytes, smem;
 };
 
@@ -441,12 +443,13 @@ int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, c
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = CLUSTER ? static_cast<unsigned>(p.splits) : 1u;
     attr[0].val.clusterDim.z = 1;
-    // Programmatic dependent launch: this kernel may start while the Z conversion before it in the stream
-    // is still finishing; it reads Zb only after griddepcontrol.wait.
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    // Programmatic dependent launch, only behind this file's own Z conversion (which is launched the
+    // ordinary way, so everything before it has completed): the kernel may then start while the conversion
+    // is finishing, pulls dY at once and reads Zb only after pdl_wait().  Behind any other kernel it is
+    // launched the ordinary way, because dY is read before the wait.
+    attr[1] = pdl_attribute();
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = p.after_conversion ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kern, tmY, tmZ, a) != cudaSuccess) {
         cudaGetLastError();
         return VELORA_ERR_CUDA;
@@ -500,6 +503,8 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
         if (rc != VELORA_OK) return rc;
     }
 
+    WgPlan plan = p;
+    plan.after_conversion = !z_in_place;
     CUtensorMap tmY, tmZ;
     rc = make_tmap_bf16_2d(&tmY, dY, O, N, lddy, 64, WG_BK);
     if (rc != VELORA_OK) return rc;
@@ -530,7 +535,7 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
 
     if (P_out) {
         // The factor alone: P = beta * P + dY^T Z (kept across micro-batches, expanded once by the caller).
-        rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, p, di.smem_optin, stream);
+        rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, plan, di.smem_optin, stream);
         if (rc != VELORA_OK) return rc;
         const int64_t total = O * p.M;
         int64_t grid = ceil_div64(total, 256);
@@ -551,8 +556,8 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
 #define VELORA_WG_CASE(LPSV, CHV)                                                                             \
         if (lps == LPSV && ch == CHV)                                                                         \
             rc = dw_dtype == VELORA_BF16                                                                      \
-                     ? launch_wg<true, LPSV, CHV, __nv_bfloat16>(tmY, tmZ, a, p, di.smem_optin, stream)       \
-                     : launch_wg<true, LPSV, CHV, float>(tmY, tmZ, a, p, di.smem_optin, stream)
+                     ? launch_wg<true, LPSV, CHV, __nv_bfloat16>(tmY, tmZ, a, plan, di.smem_optin, stream)       \
+                     : launch_wg<true, LPSV, CHV, float>(tmY, tmZ, a, plan, di.smem_optin, stream)
         VELORA_WG_CASE(1, 1);
         VELORA_WG_CASE(2, 1);
         VELORA_WG_CASE(4, 1);
@@ -565,7 +570,7 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
         if (rc == VELORA_OK) return rc;          // a refused cluster launch falls through to the three-launch route
     }
     // 2b. partial products to the workspace, then 3. dW = (sum of partials) (x) v
-    rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, p, di.smem_optin, stream);
+    rc = launch_wg<false, 1, 1, float>(tmY, tmZ, a, plan, di.smem_optin, stream);
     if (rc != VELORA_OK) return rc;
     return launch_expand_p(partials, p.splits, static_cast<int64_t>(O) * p.npad, p.npad, v, O, D, Dsub,
                            dW, dw_dtype, lddw, beta, stream);
