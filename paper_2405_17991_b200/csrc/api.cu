@@ -63,7 +63,9 @@ size_t factored_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
 {
     const size_t simt = align256(static_cast<size_t>(O) * num_subtokens(D, Dsub) * sizeof(float));
     const size_t tc = weight_grad_tc_workspace_bytes(N, D, O, Dsub);
-    return kStatusBytes + (simt > tc ? simt : tc);
+    const size_t skinny = weight_grad_skinny_workspace_bytes(N, D, O, Dsub);
+    const size_t most = simt > tc ? simt : tc;
+    return kStatusBytes + (most > skinny ? most : skinny);
 }
 
 // ---- weight gradient routing ----
@@ -77,7 +79,11 @@ int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t
     char* body = static_cast<char*>(ws) + kStatusBytes;
     if (mode == VELORA_WG_FACTORED) {
         if (ws_bytes < factored_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
-        int rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
+        // Adapter-shaped layers (O <= 64) first: too few output tiles for the tensor-core kernel to spread.
+        int rc = launch_weight_grad_skinny(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub, dW, dw_dtype, lddw,
+                                           beta, body, ws_bytes - kStatusBytes, stream, nullptr, 0);
+        if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+        rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub,
                                        dW, dw_dtype, lddw, beta, body, ws_bytes - kStatusBytes, status, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
         // CUDA-core route: P[O, M] = dY^T Z, then the outer-product expansion.
@@ -421,6 +427,11 @@ int velora_weight_grad_p(const void* dY, int dy_dtype, int64_t N, int64_t O, int
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int* status = static_cast<int*>(ws);
     char* body = static_cast<char*>(ws) + kStatusBytes;
+    if (N > 0) {
+        rc = launch_weight_grad_skinny(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, nullptr, D, Dsub, nullptr, VELORA_F32, D,
+                                       beta, body, ws_bytes - kStatusBytes, st, P, ldp);
+        if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    }
     rc = launch_weight_grad_tc(dY, dy_dtype, N, O, lddy, Z, z_dtype, ldz, nullptr, D, Dsub, nullptr, VELORA_F32, D, beta,
                                body, ws_bytes - kStatusBytes, status, st, P, ldp);
     if (rc != VELORA_ERR_UNSUPPORTED) return rc;

@@ -53,6 +53,12 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
                   float* v, void* ws, size_t ws_bytes, cudaStream_t stream, int sum_only = 0);
 // v = s / ||s|| (fp64 inside), degenerate flag read back (synchronises).
 int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
+// ---- adapter-shaped layers (skinny.cu) ----
+size_t weight_grad_skinny_workspace_bytes(int64_t N, int64_t D, int64_t O, int Dsub);
+int launch_weight_grad_skinny(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t lddy,
+                              const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
+                              void* dW, int dw_dtype, int64_t lddw, int beta,
+                              void* ws, size_t ws_bytes, cudaStream_t stream, float* P_out, int64_t ldp_out);
 size_t init_v_workspace_bytes(int Dsub);
 size_t update_v_workspace_bytes(int Dsub);
 int launch_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
