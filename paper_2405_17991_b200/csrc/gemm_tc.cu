@@ -374,6 +374,10 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
 {
     // Fused path: Dsub a power of two between 8 and 1024 (sub-token boundaries then fall on 16-byte
     // chunks of the 64-column X tiles); everything else runs the GEMM and the compress kernel in turn.
+    if (dtype == VELORA_BF16 && O <= 64) {               // adapter-shaped: one pass over X for Y and Z
+        const int src = launch_linear_forward_skinny(X, ldx, W, ldw, v, Y, ldy, Z, z_dtype, ldz, N, D, O, Dsub, status, stream);
+        if (src != VELORA_ERR_UNSUPPORTED) return src;
+    }
     const bool pow2 = Dsub >= 8 && Dsub <= VELORA_MAX_DSUB && (Dsub & (Dsub - 1)) == 0;
     const bool gemm_ok = dtype == VELORA_BF16 && N >= 1 && N < (1 << 30) && D < (1 << 30) && O < (1 << 30) &&
                          tc_operand_ok(X, ldx) && tc_operand_ok(W, ldw) && aligned16(Y) && ldy % 8 == 0;

@@ -30,6 +30,10 @@ int launch_gemm_tc_pair(int kind, const void* A, int64_t lda, const void* B, int
 int launch_linear_forward_tc_pair(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
                                   void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
                                   int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
+// Adapter-shaped layers (O <= 64): Y and Z in one pass over X.  (skinny.cu)
+int launch_linear_forward_skinny(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
+                                 void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
+                                 int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
 // True when a product with this output shape fills the device with 256 x 256 pair tiles.
 bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim);
 
