@@ -319,6 +319,22 @@ int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t
     return r == CUDA_SUCCESS ? VELORA_OK : VELORA_ERR_CUDA;
 }
 
+int make_tmap_bf16_chunks3d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
+                            int box_rows, int box_chunks)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return VELORA_ERR_CUDA;
+    if (inner % 64) return VELORA_ERR_UNSUPPORTED;
+    const cuuint64_t gdim[3] = {64, static_cast<cuuint64_t>(outer), static_cast<cuuint64_t>(inner / 64)};
+    const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(ld_elems) * 2, 128};
+    const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), static_cast<cuuint32_t>(box_chunks)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? VELORA_OK : VELORA_ERR_UNSUPPORTED;
+}
+
 bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim)
 {
     DeviceInfo di;

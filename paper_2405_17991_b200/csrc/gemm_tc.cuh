@@ -42,6 +42,12 @@ bool gemm_pair_preferred(int64_t Mdim, int64_t Ndim);
 int make_tmap_bf16_2d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
                       int box_inner, int box_outer, bool swizzle128 = true);
 bool tc_operand_ok(const void* p, int64_t ld_elems);
+// The same matrix seen as [64 elements][outer rows][inner / 64 column chunks] (inner a multiple of 64): a box of
+// box_rows rows x box_chunks chunks lands in shared memory as box_chunks tiles of box_rows x 128 bytes, each
+// swizzled like a two-dimensional 64-column box, from box_chunks * 128 contiguous bytes of every row.
+// VELORA_ERR_UNSUPPORTED if the driver does not take the description.
+int make_tmap_bf16_chunks3d(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld_elems,
+                            int box_rows, int box_chunks);
 
 // Y = X W^T with compress(X, v) computed from the same staged X tiles.
 int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,

@@ -102,29 +102,38 @@ wg_skinny_reduce_kernel(const float* __restrict__ partials, int parts, int O, in
 // the N dimension of the MMA and 64-token tiles give every SM a CTA:
 //     D[o, t] (TMEM, 128 lanes x 64 columns) += W_tile[o, k] * X_tile[t, k]      (M = 128, N = 64, K = 16)
 // Only the first O lanes of the accumulator mean anything: the A descriptor spans 128 rows of shared memory
-// but only round_up(O, 8) rows are loaded; whatever lies behind them (the next stage of the ring) feeds
-// lanes that are never read.  A stage is 8 KB of X (64 tokens x 64 columns, 128-byte swizzle) plus 1 to 8 KB
-// of W; as many stages as fit 200 KB (20 at O <= 16) keep up to 160 KB of X in flight per SM: the pass is
-// bound by HBM latency, and with 96 KB in flight it ran at 2.5 TB/s.  Warp 0 produces, warp 1 issues the MMAs, the other
-// sixteen warps compress: four sets of four warps take the sub-tokens in turn (a set needs about 0.7 us
-// for a k-block, wait and release included, and a k-block must leave every 0.2 us).  Within a set a warp
-// takes 16 of the 64 token rows, eight lanes per row read the row's eight 16-byte chunks in one instruction,
-// multiply with their slice of v and add up over the lanes of a sub-token with shuffles.  They read the X
-// tile in place and release the stage together with the MMA's commit (the kernel waits on HBM, so a stage
-// held a little longer costs nothing here).  Warps 4 and 5 finally read lanes 0..63 of the accumulator and
-// store Y.
-constexpr int SF_TOKENS = 64, SF_BK = 64, SF_MAX_STAGES = 24;
-constexpr int SF_X_BYTES = SF_TOKENS * SF_BK * 2;      // 8 KB
-constexpr int SF_RING_BYTES = 200 * 1024;              // stages of 8 KB (X) + round_up(O, 8) * 128 B (W) fill this
-constexpr int SF_BURST = 4;                            // k-blocks requested together
-constexpr int SF_SETS = 4;                             // compress warp sets (four warps each), taking sub-tokens in turn
+// but only round_up(O, 8) rows are loaded; whatever lies behind them feeds lanes that are never read.
+// A stage holds 256 columns of the 64 tokens as four 8 KB tiles (64 rows x 128 bytes, 128-byte swizzle) plus
+// the four W tiles.  Where D is a multiple of 64 ONE three-dimensional TMA box (64 elements x 64 rows x 4
+// column chunks) brings the X tiles in, 512 contiguous bytes per token row: with one box per 128-byte-wide
+// tile the same pass ran at 2.5 TB/s however deep the ring was.  Warp 0 produces, warp 1 issues the MMAs, the
+// other sixteen warps compress: four sets of four warps take the stages in turn (a sub-token that spans
+// several stages stays with one set; spreading the four tiles of a stage over the sets instead was slower,
+// every set then waking for every stage).  Within a set a warp takes 16 of the 64 token rows; eight lanes per row
+// read the row's eight 16-byte chunks of a tile in one instruction, multiply with their slice of v and add up
+// over the lanes of a sub-token with shuffles.  They read the tiles in place and release the stage together
+// with the MMA's commit (the kernel waits on HBM, so a stage held a little longer costs nothing here).  Warps 4
+// and 5 finally read lanes 0..63 of the accumulator and store Y.
+constexpr int SF_TOKENS = 64, SF_BK = 64, SF_SB = 4, SF_MAX_STAGES = 6;
+constexpr int SF_X_BYTES = SF_TOKENS * SF_BK * 2;      // 8 KB: one tile
+constexpr int SF_RING_BYTES = 200 * 1024;
+constexpr int SF_SETS = 4;                             // compress warp sets (four warps each)
 constexpr int SF_THREADS = 64 + SF_SETS * 128;
-constexpr int SF_BAR_BYTES = 2048;                     // barriers, TMEM slot, abort flag
+constexpr int SF_BAR_BYTES = 1024;                     // barriers, TMEM slot, abort flag
 constexpr size_t SF_SMEM = 1024 + SF_RING_BYTES + 16384 /* A descriptor overhang */ + SF_BAR_BYTES + VELORA_MAX_DSUB * 4;
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
 
 template <bool Z_BF16>
 __global__ void __launch_bounds__(SF_THREADS, 1)
-skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmX3,
+                      const __grid_constant__ CUtensorMap tmW, int use3d,
                       __nv_bfloat16* __restrict__ Y, int64_t ldy, int N, int O, int D, int w_rows, int stages,
                       int* __restrict__ status, const FuseArgs fz)
 {
@@ -133,12 +142,13 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     constexpr int TAIL_OFF = SF_RING_BYTES + 16384;
-    const int stage_bytes = SF_X_BYTES + ((w_rows * 128 + 1023) & ~1023);
+    const int w_tile = (w_rows * 128 + 1023) & ~1023;
+    const int stage_bytes = SF_SB * (SF_X_BYTES + w_tile);      // four X tiles, then four W tiles
     uint8_t* tail = smem + TAIL_OFF;
     const uint32_t bars = base + TAIL_OFF;
     const uint32_t full = bars, empty = bars + 8 * SF_MAX_STAGES, tfull = bars + 16 * SF_MAX_STAGES;
-    // ready[set][s]: stage s holds a landed k-block of compress set `set`.  Signalled by the MMA thread, which
-    // sees every phase of full[s] in order; a set that only looked at full[s] for its own k-blocks would skip
+    // ready[set][s]: stage s holds landed tiles for compress set `set`.  Signalled by the MMA thread, which
+    // sees every phase of full[s] in order; a set that only looked at full[s] for its own stages would skip
     // phases and could not tell them apart by parity.
     const uint32_t ready = tfull + 8;
     static_assert(8 * (2 * SF_MAX_STAGES + 1 + SF_SETS * SF_MAX_STAGES) + 16 <= SF_BAR_BYTES, "barrier area");
@@ -149,8 +159,12 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * SF_TOKENS;
     const int kblocks = (D + SF_BK - 1) / SF_BK;
+    const int nsb = (kblocks + SF_SB - 1) / SF_SB;              // stages' worth of columns
     const int cw = fz.Dsub >= SF_BK ? fz.Dsub / SF_BK : 1;      // k-blocks per sub-token (a power of two)
-    const uint32_t stage_tx = static_cast<uint32_t>(SF_X_BYTES + w_rows * 128);
+    const int cwshift = 31 - __clz(cw);
+    const uint32_t stage_tx = static_cast<uint32_t>(SF_SB * (SF_X_BYTES + w_rows * 128));
+    // The set that compresses stage-load sb: sub-tokens longer than a stage stay with one set.
+    auto set_of = [&](int sb) { return (cw > SF_SB ? (sb * SF_SB) >> cwshift : sb) & (SF_SETS - 1); };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -162,6 +176,7 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmX);
+        prefetch_tensormap(&tmX3);
         prefetch_tensormap(&tmW);
     }
     if (warp == 1) {
@@ -177,32 +192,30 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     bool failed = false;
     if (warp == 0) {
         if (lane == 0) {
-            // k-blocks are requested four at a time (the ring depth is a multiple of four): the four boxes cover
-            // 512 contiguous bytes of each token row and reach DRAM together.  One by one, 128 bytes per row
-            // and request, the same pass over X ran at 3.4 TB/s.
-            // (The host makes `stages` a multiple of four, so a burst never wraps around the ring.)
-            int it = 0;
+            int sb = 0;
             uint32_t s = 0, ph = 0;
-            while (it < kblocks && !failed) {
-                const int nb = kblocks - it < SF_BURST ? kblocks - it : SF_BURST;
-                for (int j = 0; j < nb; ++j)
-                    if (!mbar_wait(empty + 8 * (s + j), ph ^ 1u, abort_flag)) { failed = true; break; }
-                if (failed) break;
-                for (int j = 0; j < nb; ++j) {
-                    mbar_arrive_expect_tx(full + 8 * (s + j), stage_tx);
-                    const uint32_t dst = base + (s + j) * stage_bytes;
-                    tma_load_2d(dst, &tmX, full + 8 * (s + j), (it + j) * SF_BK, t0);
-                    tma_load_2d(dst + SF_X_BYTES, &tmW, full + 8 * (s + j), (it + j) * SF_BK, 0);
+            for (; sb < nsb; ++sb) {
+                if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+                mbar_arrive_expect_tx(full + 8 * s, stage_tx);
+                const uint32_t dst = base + s * stage_bytes;
+                // Column chunks beyond D are zero-filled (and counted) like any other part of a box.
+                if (use3d) {
+                    tma_load_3d(dst, &tmX3, full + 8 * s, 0, t0, sb * SF_SB);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < SF_SB; ++j)
+                        tma_load_2d(dst + j * SF_X_BYTES, &tmX, full + 8 * s, (sb * SF_SB + j) * SF_BK, t0);
                 }
-                it += nb;
-                s += nb;
-                if (s >= static_cast<uint32_t>(stages)) { s = 0; ph ^= 1u; }
+#pragma unroll
+                for (int j = 0; j < SF_SB; ++j)
+                    tma_load_2d(dst + SF_SB * SF_X_BYTES + j * w_tile, &tmW, full + 8 * s, (sb * SF_SB + j) * SF_BK, 0);
+                if (++s == static_cast<uint32_t>(stages)) { s = 0; ph ^= 1u; }
             }
             if (failed) {
                 *abort_flag = 1;
-                const int back = it < stages ? it : stages;          // own copies still in flight
+                const int back = sb < stages ? sb : stages;          // own copies still in flight
                 for (int j = 1; j <= back; ++j) {
-                    const int jt = it - j;
+                    const int jt = sb - j;
                     const unsigned long long tb = globaltimer_ns();
                     while (!mbar_try_wait(full + 8 * (jt % stages), (jt / stages) & 1u))
                         if (globaltimer_ns() - tb > kWaitLimitNs) break;
@@ -212,20 +225,23 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, SF_TOKENS, false, false);
-            const int cwshift = 31 - __clz(cw);
             uint32_t s = 0, ph = 0;
-            for (int it = 0; it < kblocks; ++it) {
+            for (int sb = 0; sb < nsb; ++sb) {
                 if (!mbar_wait(full + 8 * s, ph, abort_flag)) { failed = true; break; }
                 // Relaxed: a release in this thread would wait for the MMAs in flight.  The compress warps
                 // take their acquire from full[s] itself.
                 asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];"
-                             ::"r"(ready + 8 * (((it >> cwshift) & (SF_SETS - 1)) * SF_MAX_STAGES + s)) : "memory");
+                             ::"r"(ready + 8 * (set_of(sb) * SF_MAX_STAGES + s)) : "memory");
                 tc_fence_after_sync();
-                const uint32_t x_addr = base + s * stage_bytes, w_addr = x_addr + SF_X_BYTES;
+                const uint32_t x0 = base + s * stage_bytes, w0 = x0 + SF_SB * SF_X_BYTES;
 #pragma unroll
-                for (int j = 0; j < SF_BK / 16; ++j)
-                    umma_bf16(tmem_base, umma_smem_desc(w_addr + j * 32, 16, 1024), umma_smem_desc(x_addr + j * 32, 16, 1024),
-                              idesc, (it | j) != 0);
+                for (int j = 0; j < SF_SB; ++j) {
+                    if (sb * SF_SB + j >= kblocks) break;            // nothing but zero fill beyond D
+#pragma unroll
+                    for (int k = 0; k < SF_BK / 16; ++k)
+                        umma_bf16(tmem_base, umma_smem_desc(w0 + j * w_tile + k * 32, 16, 1024),
+                                  umma_smem_desc(x0 + j * SF_X_BYTES + k * 32, 16, 1024), idesc, (sb | j | k) != 0);
+                }
                 umma_commit(empty + 8 * s);
                 if (++s == static_cast<uint32_t>(stages)) { s = 0; ph ^= 1u; }
             }
@@ -233,71 +249,80 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             else *abort_flag = 1;
         }
     } else {
-        // ---- compress: warp cwp takes tile rows 16 cwp .. 16 cwp + 15, four at a time, eight lanes per row
+        // ---- compress: warp cwp of a set takes tile rows 16 cwp .. 16 cwp + 15, four at a time, eight lanes per row
         const int cwp = (warp - 2) & 3, set = (warp - 2) >> 2;
         const int sub = lane >> 3, c = lane & 7;
         const int lanes_per_sub = fz.Dsub >= SF_BK ? 8 : fz.Dsub / 8;      // lanes that share a sub-token inside a row
         const int dshift = 31 - __clz(fz.Dsub);
-        const int cwshift = 31 - __clz(cw);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};                                // running sums of sub-tokens longer than a k-block
-        uint32_t s = 0, ph = 0, par = 0;                         // par bit s: parity of ready[set][s]'s next phase
-        for (int it = 0; it < kblocks; ++it) {
-            if (((it >> cwshift) & (SF_SETS - 1)) != set) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};                                // running sums of sub-tokens longer than a tile
+        uint32_t s = 0, ph = 0, par = 0;                                    // par bit s: parity of ready[set][s]'s next phase
+        for (int sb = 0; sb < nsb; ++sb) {
+            if (set_of(sb) != set) {
                 if (++s == static_cast<uint32_t>(stages)) { s = 0; ph ^= 1u; }
                 continue;
             }
             if (!mbar_wait_warp(ready + 8 * (set * SF_MAX_STAGES + s), (par >> s) & 1u, abort_flag, 32)) { failed = true; break; }
             par ^= 1u << s;
-            mbar_try_wait(full + 8 * s, ph);                     // complete by now: one probe acquires the tile
-            const int jv = (((it & (cw - 1)) << 6) + c * 8) & (fz.Dsub - 1);  // position of this lane's chunk in its sub-token
-            const float4 va = *reinterpret_cast<const float4*>(sv + jv);
-            const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
-            const uint32_t tile = base + s * stage_bytes;
-            const bool last_of_sub = ((it & (cw - 1)) == cw - 1) || it == kblocks - 1;
-            // Four rows per lane, kept apart step by step (loads, products, shuffles) so that the four
-            // dependency chains overlap: a lone warp per scheduler has nothing else to hide latency with.
-            uint4 d[4];
+            mbar_try_wait(full + 8 * s, ph);                     // complete by now: one probe acquires the tiles
+            const uint32_t x0 = base + s * stage_bytes;
+            float zval[SF_SB][4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = 16 * cwp + 4 * i + sub;
-                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                             : "=r"(d[i].x), "=r"(d[i].y), "=r"(d[i].z), "=r"(d[i].w)
-                             : "r"(tile + r * 128 + (static_cast<uint32_t>(c ^ (r & 7)) << 4)));
-            }
-            float zval[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float p0 = bf16_lo(d[i].x) * va.x, p1 = bf16_hi(d[i].x) * va.y;
-                p0 = fmaf(bf16_lo(d[i].y), va.z, p0); p1 = fmaf(bf16_hi(d[i].y), va.w, p1);
-                p0 = fmaf(bf16_lo(d[i].z), vb.x, p0); p1 = fmaf(bf16_hi(d[i].z), vb.y, p1);
-                p0 = fmaf(bf16_lo(d[i].w), vb.z, p0); p1 = fmaf(bf16_hi(d[i].w), vb.w, p1);
-                zval[i] = p0 + p1;
-            }
-            for (int off = lanes_per_sub >> 1; off >= 1; off >>= 1) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) zval[i] += __shfl_xor_sync(0xffffffffu, zval[i], off);
-            }
-            if (cw > 1) {
+            for (int j = 0; j < SF_SB; ++j) {
+                const int kb = sb * SF_SB + j;
+                const int jv = (((kb & (cw - 1)) << 6) + c * 8) & (fz.Dsub - 1);   // this lane's chunk inside its sub-token
+                const float4 va = *reinterpret_cast<const float4*>(sv + jv);
+                const float4 vb = *reinterpret_cast<const float4*>(sv + jv + 4);
+                // Four rows per lane, kept apart step by step (loads, products, shuffles) so that the
+                // dependency chains overlap.
+                uint4 d[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    acc[i] += zval[i];
-                    zval[i] = acc[i];
-                    if (last_of_sub) acc[i] = 0.f;
+                    const int r = 16 * cwp + 4 * i + sub;
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(d[i].x), "=r"(d[i].y), "=r"(d[i].z), "=r"(d[i].w)
+                                 : "r"(x0 + j * SF_X_BYTES + r * 128 + (static_cast<uint32_t>(c ^ (r & 7)) << 4)));
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float p0 = bf16_lo(d[i].x) * va.x, p1 = bf16_hi(d[i].x) * va.y;
+                    p0 = fmaf(bf16_lo(d[i].y), va.z, p0); p1 = fmaf(bf16_hi(d[i].y), va.w, p1);
+                    p0 = fmaf(bf16_lo(d[i].z), vb.x, p0); p1 = fmaf(bf16_hi(d[i].z), vb.y, p1);
+                    p0 = fmaf(bf16_lo(d[i].w), vb.z, p0); p1 = fmaf(bf16_hi(d[i].w), vb.w, p1);
+                    zval[j][i] = p0 + p1;
+                }
+                for (int off = lanes_per_sub >> 1; off >= 1; off >>= 1) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) zval[j][i] += __shfl_xor_sync(0xffffffffu, zval[j][i], off);
+                }
+                if (cw > 1) {
+                    const bool last_of_sub = ((kb & (cw - 1)) == cw - 1) || kb >= kblocks - 1;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        acc[i] += zval[j][i];
+                        zval[j][i] = acc[i];
+                        if (last_of_sub) acc[i] = 0.f;
+                    }
                 }
             }
             // Release the stage BEFORE the stores to Z: the arrival is a release, and a release issued behind
-            // global stores waits until they have been performed (about a microsecond per k-block here).
-            __syncwarp();                                        // every lane's reads of the tile are done
+            // global stores waits until they have been performed.
+            __syncwarp();                                        // every lane's reads of the tiles are done
             if (lane == 0) mbar_arrive(empty + 8 * s);
-            const int m = cw == 1 ? (it * SF_BK + c * 8) >> dshift : it >> cwshift;
-            const bool writer = cw == 1 ? (c & (lanes_per_sub - 1)) == 0 : (c == 0 && last_of_sub);
-            if (writer && m < fz.M) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = t0 + 16 * cwp + 4 * i + sub;
-                    if (row < N) {
-                        if (Z_BF16) static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(zval[i]);
-                        else static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = zval[i];
+            for (int j = 0; j < SF_SB; ++j) {
+                const int kb = sb * SF_SB + j;
+                if (kb >= kblocks) break;
+                const int m = cw == 1 ? (kb * SF_BK + c * 8) >> dshift : kb >> cwshift;
+                const bool writer = cw == 1 ? (c & (lanes_per_sub - 1)) == 0
+                                            : (c == 0 && (((kb & (cw - 1)) == cw - 1) || kb == kblocks - 1));
+                if (writer && m < fz.M) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = t0 + 16 * cwp + 4 * i + sub;
+                        if (row < N) {
+                            if (Z_BF16) static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(zval[j][i]);
+                            else static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = zval[j][i];
+                        }
                     }
                 }
             }
@@ -305,7 +330,7 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         }
         if (failed) *abort_flag = 1;
         // ---- epilogue: warps 4 and 5 own TMEM lanes 0..31 and 32..63 (= output columns o)
-        if (!failed && warp >= 4 && (warp - 4) * 32 < O) {
+        if (!failed && warp >= 4 && warp <= 5 && (warp - 4) * 32 < O) {
             if (!mbar_wait_warp(tfull, 0u, abort_flag, 64)) {
                 failed = true;
                 *abort_flag = 1;
@@ -314,14 +339,14 @@ skinny_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                 const int o = (warp - 4) * 32 + lane;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>((warp - 4) * 32) << 16);
 #pragma unroll 1
-                for (int c = 0; c < SF_TOKENS / 32; ++c) {
+                for (int cc = 0; cc < SF_TOKENS / 32; ++cc) {
                     uint32_t r[32];
-                    tmem_ld_32x32(taddr + c * 32, r);
+                    tmem_ld_32x32(taddr + cc * 32, r);
                     tmem_ld_wait();
                     if (o < O) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            const int t = t0 + c * 32 + i;
+                            const int t = t0 + cc * 32 + i;
                             if (t < N) Y[static_cast<int64_t>(t) * ldy + o] = __float2bfloat16_rn(__uint_as_float(r[i]));
                         }
                     }
@@ -439,14 +464,17 @@ int launch_linear_forward_skinny(const void* X, int64_t ldx, const void* W, int6
     if (rc != VELORA_OK) return rc;
     if (static_cast<size_t>(di.smem_optin) < SF_SMEM) return VELORA_ERR_UNSUPPORTED;
     const int w_rows = static_cast<int>((O + 7) / 8 * 8);
-    const int stage_bytes = SF_X_BYTES + ((w_rows * 128 + 1023) & ~1023);
-    int stages = SF_RING_BYTES / stage_bytes / SF_BURST * SF_BURST;
+    const int w_tile = (w_rows * 128 + 1023) & ~1023;
+    int stages = SF_RING_BYTES / (SF_SB * (SF_X_BYTES + w_tile));
     if (stages > SF_MAX_STAGES) stages = SF_MAX_STAGES;
-    CUtensorMap tx, tw;
+    CUtensorMap tx, tx3, tw;
     rc = make_tmap_bf16_2d(&tx, X, D, N, ldx, SF_BK, SF_TOKENS);
     if (rc != VELORA_OK) return rc;
     rc = make_tmap_bf16_2d(&tw, W, D, O, ldw, SF_BK, w_rows);
     if (rc != VELORA_OK) return rc;
+    // One box for four 64-column tiles needs whole 64-column chunks; otherwise four two-dimensional boxes.
+    int use3d = (D % SF_BK == 0 && make_tmap_bf16_chunks3d(&tx3, X, D, N, ldx, SF_TOKENS, SF_SB) == VELORA_OK) ? 1 : 0;
+    if (!use3d) tx3 = tx;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
@@ -460,10 +488,12 @@ int launch_linear_forward_skinny(const void* X, int64_t ldx, const void* W, int6
     const int grid = static_cast<int>(ceil_div64(N, SF_TOKENS));
     if (z_dtype == VELORA_BF16)
         skinny_forward_kernel<true><<<grid, SF_THREADS, SF_SMEM, stream>>>(
-            tx, tw, static_cast<__nv_bfloat16*>(Y), ldy, static_cast<int>(N), static_cast<int>(O), static_cast<int>(D), w_rows, stages, status, fz);
+            tx, tx3, tw, use3d, static_cast<__nv_bfloat16*>(Y), ldy, static_cast<int>(N), static_cast<int>(O), static_cast<int>(D),
+            w_rows, stages, status, fz);
     else
         skinny_forward_kernel<false><<<grid, SF_THREADS, SF_SMEM, stream>>>(
-            tx, tw, static_cast<__nv_bfloat16*>(Y), ldy, static_cast<int>(N), static_cast<int>(O), static_cast<int>(D), w_rows, stages, status, fz);
+            tx, tx3, tw, use3d, static_cast<__nv_bfloat16*>(Y), ldy, static_cast<int>(N), static_cast<int>(O), static_cast<int>(D),
+            w_rows, stages, status, fz);
     return after_launch();
 }
 

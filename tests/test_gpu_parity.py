@@ -184,6 +184,42 @@ def test_forward_with_compress_inside_the_gemm(vl, N, D, O, Dsub, z_dtype):
     assert vl.velora_device_error() == 0
 
 
+ADAPTER = [
+    # N, D, O, Dsub: adapter-shaped layers (output width = adapter rank): Y and Z come from one pass over X
+    (12608, 768, 8, 32),     # ViT-B/16 adapter down-projection, rank 8
+    (2048, 4096, 16, 64),    # LoRA A on a 4096-wide projection
+    (1000, 1096, 12, 32),    # D not a multiple of 64: four two-dimensional boxes per stage instead of one
+    (777, 520, 40, 8),       # eight sub-tokens per tile, ragged tokens and columns
+    (300, 2048, 4, 256),     # a sub-token spans one stage of the ring
+    (513, 4096, 33, 1024),   # a sub-token spans four stages; O just over one TMEM lane quarter
+    (64, 64, 64, 16),        # one tile, one stage, the widest adapter
+    (130, 11008, 1, 64),     # a single output column; 172 tiles of columns = 43 stages
+]
+
+
+@pytest.mark.parametrize("N,D,O,Dsub", ADAPTER)
+@pytest.mark.parametrize("z_dtype", [torch.float32, torch.bfloat16])
+def test_adapter_shaped_layer_forward_and_backward(vl, N, D, O, Dsub, z_dtype):
+    case = vi.small_case(9500 + D + O, N, D, O, dtype="bf16", mean_offset=0.25)
+    Xa, Wa, dYa = case["X"], case["W"], case["dY"]
+    X, W = Xa.torch(DEV), Wa.torch(DEV)
+    dY = dYa.torch(DEV, ld=-(-O // 8) * 8)
+    v = vl.velora_init_v(X, Dsub)
+    v64 = to_f64(v)
+    ws = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_LINEAR_BACKWARD_FACTORED, N, D, O, Dsub), DEV)
+    for trial in range(2):                             # the second call reuses barriers' memory and TMEM
+        Y, Z = vl.velora_linear_forward(X, W, v, z_dtype=z_dtype, ws=ws)
+        assert vl.velora_workspace_status(ws) == 0
+        assert_matches(Y, oracle.linear_forward(Xa.f64(), Wa.f64()), TOL_GEMM, "Y")
+        assert_matches(Z, oracle.compress(Xa.f64(), v64), TOL_Z, "Z", ulps=1 if z_dtype == torch.bfloat16 else None)
+    dX, dW = vl.velora_linear_backward(dY, W, Z, v, ws=ws)
+    assert_matches(dX, oracle.input_grad(dYa.f64(), Wa.f64()), TOL_GEMM, "dX")
+    assert_matches(dW, oracle.weight_grad(dYa.f64(), to_f64(Z), v64, D, factored=True), TOL_GEMM, "dW")
+    P = vl.velora_weight_grad_p(dY, Z, D, Dsub, ws=ws)
+    assert_matches(vl.velora_expand_p(P, v, D), oracle.weight_grad(dYa.f64(), to_f64(Z), v64, D, factored=True), TOL_GEMM, "dW via P")
+    assert vl.velora_workspace_status(ws) == 0 and vl.velora_device_error() == 0
+
+
 def test_no_device_wait_expired_during_a_full_layer(vl):
     cfg = vi.CONFIGS[3]
     li = 0
