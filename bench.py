@@ -453,6 +453,26 @@ def kernel_table(vl, torch, L, N, ws, pk):
                 for l in [by[n] for n in ("q", "k", "v", "o")]])
     tensor("weight_grad explicit (reconstruct + GEMM dY^T Xhat)", "%dx%dx%d" % (l0["O"], N, l0["D"]), ms,
            2.0 * N * l0["D"] * l0["O"])
+    # adapter-shaped layer on the same inputs (rank-16 down-projection of an adapter on the 4096-wide stream):
+    # everything is bound by the one pass over X (forward) or over dX (input gradient)
+    R = 16
+    group = [by[n] for n in ("q", "k", "v", "o")]
+    D, M = group[0]["D"], group[0]["M"]
+    Wa = group[0]["W"][:R]                               # the first R rows of a projection serve as the adapter's A
+    Ya = torch.empty((N, R), dtype=torch.bfloat16, device=dev)
+    dYa = [l["dY"][:, :R].contiguous() for l in group]
+    dWa = torch.empty((R, D), dtype=torch.bfloat16, device=dev)
+    ws_a = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_LINEAR_BACKWARD_FACTORED, N, D, R, DSUB), dev)
+    fns = [(lambda l=l: vl.velora_linear_forward(l["X"], Wa, l["v"], Y=Ya, Z=l["Z"], ws=ws_a)) for l in group]
+    hbm("adapter forward, rank 16 (Y and Z in one pass over X)", "N=%d D=%d" % (N, D), timed(fns),
+        N * D * 2 + R * D * 2 + N * R * 2 + N * M * 4, timed_b2b(fns))
+    fns = [(lambda l=l, y=y: vl.velora_weight_grad(y, l["Z"], l["v"], D, dW=dWa, ws=ws_a)) for l, y in zip(group, dYa)]
+    hbm("adapter weight_grad factored, rank 16", "N=%d D=%d" % (N, D), timed(fns),
+        N * R * 2 + N * M * 4 + R * D * 2, timed_b2b(fns))
+    fns = [(lambda l=l, y=y: vl.velora_linear_backward(y, Wa, l["Z"], l["v"], dX=l["dX"], need_dW=False, ws=ws_a))
+           for l, y in zip(group, dYa)]
+    hbm("adapter input_grad, rank 16 (dX = dY A)", "N=%d D=%d" % (N, D), timed(fns), N * D * 2 + N * R * 2 + R * D * 2,
+        timed_b2b(fns))
     return out
 
 
