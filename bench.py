@@ -488,7 +488,7 @@ def run_profile(args):
     cfg = vi.CONFIGS[CONFIG_INDEX]
     name = {"compress": "down", "reconstruct": "down", "init_v": "down", "weight_grad": "up",
             "forward": "q", "input_grad": "q", "weight_grad_explicit": "q", "adapter_forward": "q",
-            "adapter_weight_grad": "q"}[args.profile]
+            "adapter_weight_grad": "q", "adapter_input_grad": "q"}[args.profile]
     li = [l.name for l in cfg.layers].index(name)
     layer = cfg.layers[li]
     N = cfg.N
@@ -503,12 +503,14 @@ def run_profile(args):
         fn = {"compress": lambda: vl.velora_compress(X, v, Z=Z),
               "reconstruct": lambda: vl.velora_reconstruct(Z, v, layer.D, Xhat=Xhat),
               "init_v": lambda: vl.velora_init_v(X, DSUB, v=v, ws=ws)}[args.profile]
-    elif args.profile in ("adapter_forward", "adapter_weight_grad"):      # rank-16 adapter on the q input
+    elif args.profile in ("adapter_forward", "adapter_weight_grad", "adapter_input_grad"):   # rank-16 adapter on the q input
         Wa = vi.make_W(cfg, li).torch(dev)[:16]
         dYa = vi.make_dY(cfg, li).torch(dev)[:, :16].contiguous()
         Ya = torch.empty((N, 16), dtype=torch.bfloat16, device=dev)
         dWa = torch.empty((16, layer.D), dtype=torch.bfloat16, device=dev)
+        dXa = torch.empty_like(X)
         fn = {"adapter_forward": lambda: vl.velora_linear_forward(X, Wa, v, Y=Ya, Z=Z, ws=ws),
+              "adapter_input_grad": lambda: vl.velora_linear_backward(dYa, Wa, Z, v, dX=dXa, need_dW=False, ws=ws),
               "adapter_weight_grad": lambda: vl.velora_weight_grad(dYa, Z, v, layer.D, dW=dWa, ws=ws)}[args.profile]
     else:
         W = vi.make_W(cfg, li).torch(dev)
@@ -535,7 +537,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--profile", default=None,
                     choices=["compress", "reconstruct", "init_v", "weight_grad", "weight_grad_explicit",
-                             "forward", "input_grad", "adapter_forward", "adapter_weight_grad"],
+                             "forward", "input_grad", "adapter_forward", "adapter_weight_grad", "adapter_input_grad"],
                     help="run four launches of one entry point on one layer (for ncu) and exit")
     args = ap.parse_args()
     if args.profile:
