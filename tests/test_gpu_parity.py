@@ -220,6 +220,27 @@ def test_adapter_shaped_layer_forward_and_backward(vl, N, D, O, Dsub, z_dtype):
     assert vl.velora_workspace_status(ws) == 0 and vl.velora_device_error() == 0
 
 
+def test_adapter_shaped_gradient_accumulation(vl):
+    """beta = 1 on the adapter-shaped weight-gradient path: dW += ..., and P accumulated over two micro-batches."""
+    N, D, O, Dsub = 900, 768, 24, 32
+    case = vi.small_case(9700, N, D, O, dtype="bf16", mean_offset=0.25)
+    X, dY = case["X"].torch(DEV), case["dY"].torch(DEV)
+    v = vl.velora_init_v(X, Dsub)
+    Z = vl.velora_compress(X, v)
+    v64, Z64, dY64 = to_f64(v), to_f64(Z), case["dY"].f64()
+    base = torch.randn(O, D, device=DEV, generator=torch.Generator(DEV).manual_seed(6))
+    for dt in (torch.float32, torch.bfloat16):
+        dW = base.to(dt).clone()
+        vl.velora_weight_grad(dY, Z, v, D, dW=dW, beta=1)
+        ref = oracle.weight_grad(dY64, Z64, v64, D, dW0=to_f64(base.to(dt)))
+        assert_matches(dW, ref, TOL_GEMM, "dW accumulate, adapter-shaped")
+    cut = 333
+    P = vl.velora_weight_grad_p(dY[:cut], Z[:cut], D, Dsub)
+    vl.velora_weight_grad_p(dY[cut:], Z[cut:], D, Dsub, P=P, beta=1)
+    assert_matches(vl.velora_expand_p(P, v, D, dw_dtype=torch.float32), oracle.weight_grad(dY64, Z64, v64, D, factored=True),
+                   TOL_GEMM, "dW from P over two micro-batches")
+
+
 def test_no_device_wait_expired_during_a_full_layer(vl):
     cfg = vi.CONFIGS[3]
     li = 0
