@@ -299,31 +299,54 @@ def run_ours(args):
     if rank == 0:
         line["kernels"] = kernel_table(vl, torch, L, N, ws, pk)
 
-    # ---- end to end: host buffers in, gradients out, through velora_linear_step_host
+    # ---- end to end: host buffers in, gradients out, through velora_linear_step_host.  Three streams, each
+    # with its own staging area and workspace, take the layers in turn, so that one layer's copies from and
+    # to the host overlap the neighbouring layers' kernels (the copies dominate: 1.28 GB in, 0.40 GB out).
     e2e_steps = max(1, min(args.steps, 5))
+    n_streams = 3
     staging_bytes = max(vl.velora_host_step_staging_bytes(N, l["D"], l["O"], DSUB) for l in L)
-    staging = torch.empty(staging_bytes, dtype=torch.uint8, device=dev)
+    lanes = []
+    for _ in range(n_streams):
+        w = vl.velora_workspace_alloc(ws.numel(), dev)
+        lanes.append({"stream": torch.cuda.Stream(device=dev), "staging": torch.empty(staging_bytes, dtype=torch.uint8, device=dev),
+                      "ws": w, "done": torch.cuda.Event()})
     for l in L:
         l["hdW"] = torch.empty((l["O"], l["D"]), dtype=torch.bfloat16).pin_memory()
+    torch.cuda.synchronize(dev)
 
-    def host_step():
-        for l in L:
-            vl.velora_linear_step_host(l["hX"], l["hdY"], l["W"], l["v"], staging, ws, hdW=l["hdW"])
+    def host_steps(count):
+        """`count` steps; returns after the current stream has been made to wait for all of them."""
+        start = torch.cuda.Event()
+        start.record()
+        for ln in lanes:
+            ln["stream"].wait_event(start)
+        i = 0
+        for _ in range(count):
+            for l in L:
+                ln = lanes[i % n_streams]
+                i += 1
+                vl.velora_linear_step_host(l["hX"], l["hdY"], l["W"], l["v"], ln["staging"], ln["ws"], hdW=l["hdW"],
+                                           stream=ln["stream"])
+        for ln in lanes:
+            ln["done"].record(ln["stream"])
+            torch.cuda.current_stream().wait_event(ln["done"])
 
-    host_step()
+    host_steps(1)
     barrier()
     s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s2.record()
-    for _ in range(e2e_steps):
-        host_step()
+    host_steps(e2e_steps)
     e2.record()
     barrier()
+    for ln in lanes:
+        if vl.velora_workspace_status(ln["ws"]) != 0:
+            raise RuntimeError("device status raised during the end-to-end steps")
     e2e_ms, e2e_tokens = aggregate_over_ranks(s2.elapsed_time(e2), N * e2e_steps, dist if world > 1 else None, dev)
     line["e2e"] = {
         "value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
         "h2d_bytes_per_step": int(sum(N * (l["D"] + l["O"]) * 2 for l in L)),
         "d2h_bytes_per_step": int(sum(l["O"] * l["D"] * 2 for l in L)),
-        "api": "velora_linear_step_host (pinned host X, dY in; dW out)",
+        "api": "velora_linear_step_host (pinned host X, dY in; dW out), layers dealt round-robin to %d streams" % n_streams,
     }
 
     if rank == 0:
