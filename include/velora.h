@@ -186,6 +186,10 @@ int velora_weight_grad(const void* dY, int dy_dtype, int64_t N, int64_t O, int64
  * `dtype` is the storage type of X, W and Y (bf16: tensor cores with fp32
  * accumulation; f32: CUDA cores).  Z as in velora_compress.  X itself need not
  * be kept by the caller afterwards: (Z, W, v) is all the backward needs.
+ * With bf16 data, 16-byte aligned rows and Dsub a power of two in 8 .. 1024, X is read
+ * from HBM once for both results: inside the tensor-core product for wide layers
+ * (O > 768), in a single streaming pass for adapter-shaped ones (O <= 64, Section 4:
+ * down projections of adapters); other shapes run the product and then velora_compress.
  * ws: velora_workspace_bytes(VELORA_OP_LINEAR_FORWARD, ...) bytes.
  */
 int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* v,
