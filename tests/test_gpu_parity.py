@@ -194,6 +194,9 @@ ADAPTER = [
     (513, 4096, 33, 1024),   # a sub-token spans four stages; O just over one TMEM lane quarter
     (64, 64, 64, 16),        # one tile, one stage, the widest adapter
     (130, 11008, 1, 64),     # a single output column; 172 tiles of columns = 43 stages
+    (500, 1024, 24, 128),    # 17..32 output columns: four-stage ring
+    (1, 256, 8, 64),         # a single token
+    (65, 128, 20, 32),       # one token beyond a tile
     (8192, 4096, 16, 64),    # the benchmark's adapter row at full size
     (8192, 11008, 64, 256),  # full-size down-projection input, widest adapter, sub-token = one stage
 ]
