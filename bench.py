@@ -273,6 +273,28 @@ def run_ours(args):
         barrier()
     elapsed_ms = start.elapsed_time(end)
     launches = vl.velora_launch_count() - launches0
+    graph_ms = None
+    if args.graph:
+        # The same step captured once into a CUDA graph and replayed: what a launch-bound configuration gains
+        # when the host submits one graph instead of 4-5 kernels per layer.  Reported beside the plain figure.
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        for _ in range(3):
+            g.replay()
+        barrier()
+        gs, ge = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        gs.record()
+        for _ in range(args.steps):
+            g.replay()
+        ge.record()
+        barrier()
+        graph_ms = gs.elapsed_time(ge) / args.steps
     status = vl.velora_workspace_status(ws)
     if status != 0:
         raise RuntimeError("device status %d (%s) after the timed region" % (status, vl.velora_status_string(status)))
@@ -304,6 +326,9 @@ def run_ours(args):
         "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg), "clocks": clocks.summary(),
         "gpu_launches": int(launches), "roofline": roofline,
     }
+    if graph_ms is not None:
+        line["cuda_graph"] = {"ms_per_step": graph_ms, "value": N * world / (graph_ms * 1e-3), "unit": UNIT,
+                              "note": "the same step replayed from one captured graph (this rank's time)"}
 
     if not full:                                   # a parity-test configuration timed on request: the step only
         if rank == 0:
@@ -581,6 +606,8 @@ def main():
     ap.add_argument("--config", type=int, default=CONFIG_DEFAULT, choices=[2, 3, 4, 5],
                     help="time the step of another configuration (its first sub-token length); the headline line, "
                          "the kernel table and the end-to-end leg are configuration 5's")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the step replayed from a CUDA graph (an extra key; the headline stays the plain step)")
     args = ap.parse_args()
     global CONFIG_INDEX, DSUB
     if args.config != CONFIG_DEFAULT:

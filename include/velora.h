@@ -21,7 +21,12 @@
  *     dW = dY^T Xhat.  The listing in Algorithm 1 is only consistent with
  *     this layout.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
- *     Work is enqueued asynchronously; only velora_init_v synchronises.
+ *     Work is enqueued asynchronously; only velora_init_v, velora_normalize_v and the
+ *     two status readers synchronise.  The asynchronous entry points use nothing but
+ *     kernel launches (and, for the host-buffer step, asynchronous copies) on `stream`,
+ *     so after one ordinary call per shape (which sets the kernels' shared-memory
+ *     limits on that device) a sequence of them can be captured into a CUDA graph:
+ *     the forward + backward of a layer replayed from a graph gives the same bits.
  *   - Return value: a velora_status.  Arguments are validated on the host
  *     before anything is launched; on a non-zero status no output is written
  *     (VELORA_ERR_CUDA and VELORA_ERR_TIMEOUT excepted, which report a failure

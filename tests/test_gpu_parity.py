@@ -246,6 +246,44 @@ def test_adapter_shaped_gradient_accumulation(vl):
                    TOL_GEMM, "dW from P over two micro-batches")
 
 
+def test_a_layer_replayed_from_a_cuda_graph_gives_the_same_bits(vl):
+    """Forward + backward captured once (after a warm-up call) and replayed: identical results, no device error."""
+    cfg = vi.CONFIGS[2]
+    for li in (0, 4):                                  # q (product then compress) and up (compress inside the product)
+        X, W, dY = vi.make_X(cfg, li).torch(DEV), vi.make_W(cfg, li).torch(DEV), vi.make_dY(cfg, li).torch(DEV)
+        N, D = X.shape
+        O = W.shape[0]
+        ws = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_LINEAR_BACKWARD_FACTORED, N, D, O, 64), DEV)
+        v = vl.velora_init_v(X, 64)
+        out = {k: torch.empty(shape, device=DEV, dtype=dt) for k, shape, dt in
+               (("Y", (N, O), torch.bfloat16), ("Z", (N, D // 64), torch.float32), ("dX", (N, D), torch.bfloat16),
+                ("dW", (O, D), torch.bfloat16))}
+
+        def layer():
+            vl.velora_linear_forward(X, W, v, Y=out["Y"], Z=out["Z"], ws=ws)
+            vl.velora_linear_backward(dY, W, out["Z"], v, dX=out["dX"], dW=out["dW"], ws=ws)
+
+        layer()
+        torch.cuda.synchronize()
+        eager = {k: t.clone() for k, t in out.items()}
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            layer()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            layer()
+        for t in out.values():
+            t.zero_()
+        g.replay()
+        g.replay()
+        torch.cuda.synchronize()
+        for k in out:
+            assert torch.equal(out[k], eager[k]), k
+        assert vl.velora_workspace_status(ws) == 0 and vl.velora_device_error() == 0
+
+
 def test_no_device_wait_expired_during_a_full_layer(vl):
     cfg = vi.CONFIGS[3]
     li = 0
