@@ -1,11 +1,15 @@
 // Adapter-shaped layers (Section 4: VeLoRA on the down projections of trainable adapters, output width
-// O = the adapter rank, 4 .. 64): the factored weight gradient of Algorithm 1 for a tiny O.
+// O = the adapter rank, 4 .. 64).  Two things live here, both from Algorithm 1 with a tiny O:
+//
+//  1. the factored weight gradient
 //     P[o, m] = sum_n dY[n, o] * Z[n, m]            (O x M <= 64 x 256 values, a few MFLOP)
 //     dW[o, m*Dsub + j] = beta*dW + P[o, m] * v[j]
 // With one or two output tiles the tensor-core kernel of weight_grad_tc.cu cannot spread over the SMs (at
-// most 8 CTAs pull on dY and Z); here every SM takes a slice of the tokens and forms its own partial P on
-// the CUDA cores, a second kernel adds the partials in a fixed order, and the common expansion kernel
-// writes dW.  All sums are fp32, products are formed from the stored values (Z is not rounded to bf16).
+// most 8 CTAs pull on dY and Z); here the tokens are cut into up to 512 slices, each CTA forms the partial P of
+// its slice on the CUDA cores, a second kernel adds the partials in a fixed order, and the common expansion
+// kernel writes dW.  All sums are fp32, products are formed from the stored values (Z is not rounded to bf16).
+//
+//  2. the forward, Y = X W^T and Z = compress(X, v) in one pass over X (further down).
 #include "common.cuh"
 #include "gemm_fuse.cuh"
 #include "gemm_tc.cuh"
