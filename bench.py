@@ -51,7 +51,7 @@ def peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
