@@ -368,6 +368,19 @@ def test_results_are_run_to_run_identical(vl):
     # a frozen v survives a save / reload: Z is bit-identical
     v2 = outs[0][0].cpu().clone().to(DEV)
     assert torch.equal(vl.velora_compress(X, v2), vl.velora_compress(X, outs[0][0]))
+    # the adapter-shaped kernels (sliced partial sums, compress warp sets) and the large clustered and paired ones
+    for (N, D, O, Dsub) in ((8192, 4096, 16, 64), (4096, 4096, 4096, 64)):
+        case = vi.small_case(41 + O, N, D, O, dtype="bf16", mean_offset=0.1)
+        X, W, dY = case["X"].torch(DEV), case["W"].torch(DEV), case["dY"].torch(DEV)
+        v = vl.velora_init_v(X, Dsub)
+        outs = []
+        for _ in range(3):
+            Y, Z = vl.velora_linear_forward(X, W, v)
+            dX, dW = vl.velora_linear_backward(dY, W, Z, v)
+            outs.append((Y, Z, dX, dW))
+        for other in outs[1:]:
+            for a, b in zip(outs[0], other):
+                assert torch.equal(a, b)
 
 
 # ------------------------------------------------------------------ weight gradient and dense products
