@@ -411,6 +411,89 @@ expand_p_elem_kernel(const float* __restrict__ P, int splits, int64_t split_stri
     }
 }
 
+// ------------------------------------------------------------------ sub-tokens shorter than a 16-byte chunk
+// Dsub in {1, 2, 4} (the paper's smallest setting, sub-token length 4 with rank-4 adapters): a 16-byte chunk of
+// a row holds 8 / Dsub whole sub-tokens, so a thread needs no partner: one 128-bit load, 8 / Dsub dot
+// products (compress) or 8 / Dsub scalars times v (reconstruct), coalesced stores.  Four chunks per thread are
+// in flight.  Columns beyond D inside the last chunk of a row (row pitch padded to 8) are treated as zeros.
+template <int DS, typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+compress_small_kernel(const uint4* __restrict__ X, int64_t N, int D, int64_t ldc, int M,
+                      const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz)
+{
+    constexpr int PER = 8 / DS;
+    float vr[DS];
+#pragma unroll
+    for (int j = 0; j < DS; ++j) vr[j] = __ldg(v + j);
+    const int chunks = (D + 7) / 8;
+    const int64_t total = N * chunks;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; base < total; base += 4 * stride) {
+        uint4 d[4];
+        int64_t row[4];
+        int c[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t idx = base + u * stride;
+            row[u] = idx / chunks;
+            c[u] = static_cast<int>(idx - row[u] * chunks);
+            d[u] = idx < total ? __ldg(X + row[u] * ldc + c[u]) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (base + u * stride >= total) break;
+            float x[8];
+            x[0] = bf16_lo(d[u].x); x[1] = bf16_hi(d[u].x);
+            x[2] = bf16_lo(d[u].y); x[3] = bf16_hi(d[u].y);
+            x[4] = bf16_lo(d[u].z); x[5] = bf16_hi(d[u].z);
+            x[6] = bf16_lo(d[u].w); x[7] = bf16_hi(d[u].w);
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                if (8 * c[u] + e >= D) x[e] = 0.f;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                float z = 0.f;
+#pragma unroll
+                for (int j = 0; j < DS; ++j) z = fmaf(x[k * DS + j], vr[j], z);
+                const int m = c[u] * PER + k;
+                if (m < M) Elem<ZT>::store(Z + row[u] * ldz + m, z);
+            }
+        }
+    }
+}
+
+template <int DS, typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+reconstruct_small_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D, int M,
+                         const float* __restrict__ v, uint4* __restrict__ Xhat, int64_t ldc)
+{
+    constexpr int PER = 8 / DS;
+    float vr[DS];
+#pragma unroll
+    for (int j = 0; j < DS; ++j) vr[j] = __ldg(v + j);
+    const int chunks = (D + 7) / 8;                       // D is a multiple of 8 here (whole 16-byte stores)
+    const int64_t total = N * chunks;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; idx < total; idx += stride) {
+        const int64_t row = idx / chunks;
+        const int c = static_cast<int>(idx - row * chunks);
+        float y[8];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            const int m = c * PER + k;
+            const float z = m < M ? Elem<ZT>::load(Z + row * ldz + m) : 0.f;
+#pragma unroll
+            for (int j = 0; j < DS; ++j) y[k * DS + j] = z * vr[j];
+        }
+        uint4 o;
+        o.x = pack_bf16x2(y[0], y[1]);
+        o.y = pack_bf16x2(y[2], y[3]);
+        o.z = pack_bf16x2(y[4], y[5]);
+        o.w = pack_bf16x2(y[6], y[7]);
+        __stcs(Xhat + row * ldc + c, o);
+    }
+}
+
 // ------------------------------------------------------------------ host side
 struct VecShape {
     bool ok;
@@ -592,6 +675,21 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
         const int rc = launch_compress_tma(X, N, D, ldx, Dsub, v, Z, z_dtype, ldz, nullptr, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     }
+    if (x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && rows_vectorisable(X, ldx) && D < (1 << 30)) {
+        int grid = 0;
+        const int rc = stream_grid(N * ceil_div64(D, 8), 4, &grid);
+        if (rc != VELORA_OK) return rc;
+#define CALL_SMALL(DSV)                                                                                     \
+        if (z_dtype == VELORA_F32)                                                                          \
+            compress_small_kernel<DSV, float><<<grid, kStreamThreads, 0, stream>>>(                         \
+                static_cast<const uint4*>(X), N, static_cast<int>(D), ldx / 8, M, v, static_cast<float*>(Z), ldz); \
+        else                                                                                                \
+            compress_small_kernel<DSV, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(                 \
+                static_cast<const uint4*>(X), N, static_cast<int>(D), ldx / 8, M, v, static_cast<__nv_bfloat16*>(Z), ldz)
+        if (Dsub == 1) { CALL_SMALL(1); } else if (Dsub == 2) { CALL_SMALL(2); } else { CALL_SMALL(4); }
+#undef CALL_SMALL
+        return check_launch();
+    }
     if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx)) {
         const int64_t step = max_rows_per_launch(M * vs.lps, ldx / 8, ldz);
         const int d = static_cast<int>(D), ldc = static_cast<int>(ldx / 8), ldzi = static_cast<int>(ldz);
@@ -639,6 +737,23 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
     if (x_dtype == VELORA_BF16) {                        // Xhat = Z (x) v is the one-split, beta = 0 expansion
         const int rc = launch_expand_rows_vec(Z, z_dtype, 1, 0, ldz, v, N, D, Dsub, Xhat, x_dtype, ldxhat, 0, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    }
+    if (x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && D % 8 == 0 && rows_vectorisable(Xhat, ldxhat) &&
+        D < (1 << 30)) {
+        const int M = static_cast<int>(ceil_div64(D, Dsub));
+        int grid = 0;
+        const int rc = stream_grid(N * (D / 8), 1, &grid);
+        if (rc != VELORA_OK) return rc;
+#define CALL_SMALL(DSV)                                                                                     \
+        if (z_dtype == VELORA_F32)                                                                          \
+            reconstruct_small_kernel<DSV, float><<<grid, kStreamThreads, 0, stream>>>(                      \
+                static_cast<const float*>(Z), ldz, N, static_cast<int>(D), M, v, static_cast<uint4*>(Xhat), ldxhat / 8); \
+        else                                                                                                \
+            reconstruct_small_kernel<DSV, __nv_bfloat16><<<grid, kStreamThreads, 0, stream>>>(              \
+                static_cast<const __nv_bfloat16*>(Z), ldz, N, static_cast<int>(D), M, v, static_cast<uint4*>(Xhat), ldxhat / 8)
+        if (Dsub == 1) { CALL_SMALL(1); } else if (Dsub == 2) { CALL_SMALL(2); } else { CALL_SMALL(4); }
+#undef CALL_SMALL
+        return check_launch();
     }
     int grid = 0;
     int rc = stream_grid(N * D, 4, &grid);

@@ -121,6 +121,10 @@ EDGE = [
     (130, 2048, 16, 1024), # longest supported sub-token
     (1000, 40, 33, 8),     # one chunk per sub-token
     (257, 136, 130, 10),   # Dsub not a multiple of 8
+    (1000, 768, 40, 4),    # the paper's shortest sub-tokens: two per 16-byte chunk
+    (300, 260, 24, 2),     # four per chunk; D not a multiple of 8 (last chunk half real)
+    (257, 104, 16, 1),     # eight per chunk
+    (500, 99, 12, 4),      # ragged last sub-token (3 of 4) inside the last chunk
 ]
 
 
