@@ -494,6 +494,142 @@ reconstruct_small_kernel(const ZT* __restrict__ Z, int64_t ldz, int64_t N, int D
     }
 }
 
+// ------------------------------------------------------------------ any sub-token length that is a multiple of 8
+// The paper's sub-token size ablation uses D/8 .. D/64 of a 768-wide layer: 96, 48, 24 (Section 5), none a
+// power of two.  compress: a warp walks a row in windows of 32 chunks (512 contiguous bytes per load
+// instruction); a lane multiplies its chunk with its slice of v, then the lanes of a sub-token are added up
+// by a segmented shuffle reduction (the key is the sub-token index), and what a sub-token has collected when
+// the window ends is carried into the next window by the same warp.  Sums run in a fixed order.
+template <typename ZT>
+__global__ void __launch_bounds__(kStreamThreads)
+compress_seg_kernel(const uint4* __restrict__ X, int N, int D, int64_t ldc, int Dsub, int M,
+                    const float* __restrict__ v, ZT* __restrict__ Z, int64_t ldz)
+{
+    extern __shared__ float sv_seg[];
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) sv_seg[j] = __ldg(v + j);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int chunks = (D + 7) / 8;
+    const int warps = gridDim.x * (kStreamThreads / 32);
+    for (int row = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5); row < N; row += warps) {
+        const uint4* xr = X + static_cast<int64_t>(row) * ldc;
+        float carry = 0.f;
+        int carry_m = -1;
+        for (int w0 = 0; w0 < chunks; w0 += 128) {          // four windows (2 KB of the row) in flight
+            uint4 d[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = w0 + 32 * u + lane;
+                d[u] = c < chunks ? __ldg(xr + c) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int wbase = w0 + 32 * u;
+                if (wbase >= chunks) break;
+                const int c = wbase + lane;
+                const bool valid = c < chunks;
+                const int m = valid ? (8 * c) / Dsub : -2 - lane;
+                float p = 0.f;
+                if (valid) {
+                    const int j0 = 8 * c - m * Dsub;
+                    const float4 va = *reinterpret_cast<const float4*>(sv_seg + j0);
+                    const float4 vb = *reinterpret_cast<const float4*>(sv_seg + j0 + 4);
+                    float x[8];
+                    x[0] = bf16_lo(d[u].x); x[1] = bf16_hi(d[u].x);
+                    x[2] = bf16_lo(d[u].y); x[3] = bf16_hi(d[u].y);
+                    x[4] = bf16_lo(d[u].z); x[5] = bf16_hi(d[u].z);
+                    x[6] = bf16_lo(d[u].w); x[7] = bf16_hi(d[u].w);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (8 * c + e >= D) x[e] = 0.f;              // padding of the row pitch is not data
+                    p = x[0] * va.x;
+                    p = fmaf(x[1], va.y, p); p = fmaf(x[2], va.z, p); p = fmaf(x[3], va.w, p);
+                    p = fmaf(x[4], vb.x, p); p = fmaf(x[5], vb.y, p); p = fmaf(x[6], vb.z, p); p = fmaf(x[7], vb.w, p);
+                }
+                // After the five steps the first lane of every run of equal keys holds the run's sum.
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const float p2 = __shfl_down_sync(0xffffffffu, p, off);
+                    const int m2 = __shfl_down_sync(0xffffffffu, m, off);
+                    if (lane + off < 32 && m2 == m) p += p2;
+                }
+                const int m_left = __shfl_up_sync(0xffffffffu, m, 1);
+                const bool head = valid && (lane == 0 || m_left != m);
+                if (lane == 0 && m == carry_m) p += carry;           // the sub-token began in an earlier window
+                // Last chunk of sub-token m: the one before the next sub-token starts, or the row's last chunk.
+                int end_chunk = ((m + 1) * Dsub) / 8 - 1;
+                if (end_chunk > chunks - 1) end_chunk = chunks - 1;
+                const bool ends_here = end_chunk <= wbase + 31;
+                if (head && ends_here && m < M) Elem<ZT>::store(Z + static_cast<int64_t>(row) * ldz + m, p);
+                const unsigned heads = __ballot_sync(0xffffffffu, head);
+                const int last_head = 31 - __clz(heads);             // heads != 0: lane 0 of a live window is valid
+                const float p_last = __shfl_sync(0xffffffffu, p, last_head);
+                const int m_last = __shfl_sync(0xffffffffu, m, last_head);
+                const int open = __shfl_sync(0xffffffffu, ends_here ? 0 : 1, last_head);
+                carry = p_last;
+                carry_m = open ? m_last : -1;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void store8(__nv_bfloat16* p, float (&y)[8], int beta)
+{
+    uint4* q = reinterpret_cast<uint4*>(p);
+    if (beta) {
+        const uint4 old = *q;
+        y[0] += bf16_lo(old.x); y[1] += bf16_hi(old.x);
+        y[2] += bf16_lo(old.y); y[3] += bf16_hi(old.y);
+        y[4] += bf16_lo(old.z); y[5] += bf16_hi(old.z);
+        y[6] += bf16_lo(old.w); y[7] += bf16_hi(old.w);
+    }
+    uint4 o;
+    o.x = pack_bf16x2(y[0], y[1]);
+    o.y = pack_bf16x2(y[2], y[3]);
+    o.z = pack_bf16x2(y[4], y[5]);
+    o.w = pack_bf16x2(y[6], y[7]);
+    __stcs(q, o);
+}
+__device__ __forceinline__ void store8(float* p, float (&y)[8], int beta)
+{
+    float4* q = reinterpret_cast<float4*>(p);
+    if (beta) {
+        const float4 a = q[0], b = q[1];
+        y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
+        y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
+    }
+    __stcs(q, make_float4(y[0], y[1], y[2], y[3]));
+    __stcs(q + 1, make_float4(y[4], y[5], y[6], y[7]));
+}
+
+// out[r, 8c .. 8c+7] = beta * out + (sum_s S[s][r][m(c)]) * v[...]: one thread per 16-byte-aligned group of eight
+// outputs, for any Dsub that is a multiple of 8 (a group then lies inside one sub-token).  Serves reconstruct
+// (one split, beta = 0) and the expansion of the factor P where the power-of-two kernel does not apply.
+template <typename ST, typename WT>
+__global__ void __launch_bounds__(kStreamThreads)
+expand_any_kernel(const ST* __restrict__ S, int splits, int64_t split_stride, int64_t lds, const float* __restrict__ v,
+                  int64_t R, int D, int Dsub, WT* __restrict__ out, int64_t ldo, int beta)
+{
+    extern __shared__ float sv_any[];
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) sv_any[j] = __ldg(v + j);
+    __syncthreads();
+    const int chunks = D / 8;                                 // D is a multiple of 8 here
+    const int64_t total = R * chunks;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; idx < total; idx += stride) {
+        const int64_t r = idx / chunks;
+        const int c = static_cast<int>(idx - r * chunks);
+        const int m = (8 * c) / Dsub;
+        const int j0 = 8 * c - m * Dsub;
+        float z = 0.f;
+        for (int sp = 0; sp < splits; ++sp) z += Elem<ST>::load(S + sp * split_stride + r * lds + m);   // fixed order
+        const float4 va = *reinterpret_cast<const float4*>(sv_any + j0);
+        const float4 vb = *reinterpret_cast<const float4*>(sv_any + j0 + 4);
+        float y[8] = {z * va.x, z * va.y, z * va.z, z * va.w, z * vb.x, z * vb.y, z * vb.z, z * vb.w};
+        store8(out + r * ldo + 8 * c, y, beta);                // 16-byte aligned: checked on the host
+    }
+}
+
 // ------------------------------------------------------------------ host side
 struct VecShape {
     bool ok;
@@ -717,6 +853,21 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
         }
         return VELORA_OK;
     }
+    if (x_dtype == VELORA_BF16 && Dsub % 8 == 0 && rows_vectorisable(X, ldx) && N < (1 << 30) && D < (1 << 28)) {
+        // any other multiple of 8 (96, 48, 24 ...): segmented reduction over the lanes of a sub-token
+        int sgrid = 0;
+        const int src = stream_grid(N * 32, 1, &sgrid);
+        if (src != VELORA_OK) return src;
+        const size_t smem = static_cast<size_t>(Dsub) * sizeof(float);
+        if (z_dtype == VELORA_F32)
+            compress_seg_kernel<float><<<sgrid, kStreamThreads, smem, stream>>>(
+                static_cast<const uint4*>(X), static_cast<int>(N), static_cast<int>(D), ldx / 8, Dsub, M, v, static_cast<float*>(Z), ldz);
+        else
+            compress_seg_kernel<__nv_bfloat16><<<sgrid, kStreamThreads, smem, stream>>>(
+                static_cast<const uint4*>(X), static_cast<int>(N), static_cast<int>(D), ldx / 8, Dsub, M, v,
+                static_cast<__nv_bfloat16*>(Z), ldz);
+        return check_launch();
+    }
     int grid = 0;
     int rc = stream_grid(N * M * 32, 1, &grid);
     if (rc != VELORA_OK) return rc;
@@ -728,6 +879,31 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
     else if (z_dtype == VELORA_F32) CALL_ELEM(float, float);
     else CALL_ELEM(float, __nv_bfloat16);
 #undef CALL_ELEM
+    return check_launch();
+}
+
+// Per-chunk expansion for any Dsub that is a multiple of 8; VELORA_ERR_UNSUPPORTED (nothing launched) otherwise.
+static int launch_expand_any(const void* S, int s_dtype, int splits, int64_t split_stride, int64_t lds, const float* v,
+                             int64_t R, int64_t D, int Dsub, void* out, int out_dtype, int64_t ldo, int beta,
+                             cudaStream_t stream)
+{
+    if (Dsub % 8 || D % 8 || D >= (1 << 28) || R < 1) return VELORA_ERR_UNSUPPORTED;
+    if (!aligned16(out) || (ldo * static_cast<int64_t>(dtype_size(out_dtype))) % 16) return VELORA_ERR_UNSUPPORTED;
+    if (s_dtype == VELORA_BF16 && out_dtype != VELORA_BF16) return VELORA_ERR_UNSUPPORTED;
+    int grid = 0;
+    const int rc = stream_grid(R * (D / 8), 2, &grid);
+    if (rc != VELORA_OK) return rc;
+    const size_t smem = static_cast<size_t>(Dsub) * sizeof(float);
+    const int d = static_cast<int>(D);
+    if (s_dtype == VELORA_BF16)
+        expand_any_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, kStreamThreads, smem, stream>>>(
+            static_cast<const __nv_bfloat16*>(S), splits, split_stride, lds, v, R, d, Dsub, static_cast<__nv_bfloat16*>(out), ldo, beta);
+    else if (out_dtype == VELORA_BF16)
+        expand_any_kernel<float, __nv_bfloat16><<<grid, kStreamThreads, smem, stream>>>(
+            static_cast<const float*>(S), splits, split_stride, lds, v, R, d, Dsub, static_cast<__nv_bfloat16*>(out), ldo, beta);
+    else
+        expand_any_kernel<float, float><<<grid, kStreamThreads, smem, stream>>>(
+            static_cast<const float*>(S), splits, split_stride, lds, v, R, d, Dsub, static_cast<float*>(out), ldo, beta);
     return check_launch();
 }
 
@@ -755,6 +931,10 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
 #undef CALL_SMALL
         return check_launch();
     }
+    {
+        const int arc = launch_expand_any(Z, z_dtype, 1, 0, ldz, v, N, D, Dsub, Xhat, x_dtype, ldxhat, 0, stream);
+        if (arc != VELORA_ERR_UNSUPPORTED) return arc;
+    }
     int grid = 0;
     int rc = stream_grid(N * D, 4, &grid);
     if (rc != VELORA_OK) return rc;
@@ -774,6 +954,8 @@ int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ld
                     cudaStream_t stream)
 {
     int rc = launch_expand_rows_vec(P, VELORA_F32, splits, split_stride, ldp, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    rc = launch_expand_any(P, VELORA_F32, splits, split_stride, ldp, v, O, D, Dsub, dW, dw_dtype, lddw, beta, stream);
     if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     int grid = 0;
     rc = stream_grid(O * D, 4, &grid);

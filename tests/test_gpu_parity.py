@@ -121,6 +121,11 @@ EDGE = [
     (130, 2048, 16, 1024), # longest supported sub-token
     (1000, 40, 33, 8),     # one chunk per sub-token
     (257, 136, 130, 10),   # Dsub not a multiple of 8
+    (1000, 768, 48, 96),   # the sub-token sizes of the paper's ablation on a 768-wide layer: D/8 ...
+    (1000, 768, 40, 48),   # ... D/16 ...
+    (700, 768, 24, 24),    # ... D/32: none a power of two (segmented reduction, per-chunk expansion)
+    (333, 1000, 56, 40),   # sub-tokens straddling the 32-chunk windows of a row, D not a multiple of Dsub
+    (200, 4096, 32, 1000), # a sub-token longer than three windows; ragged last one (96 of 1000)
     (1000, 768, 40, 4),    # the paper's shortest sub-tokens: two per 16-byte chunk
     (300, 260, 24, 2),     # four per chunk; D not a multiple of 8 (last chunk half real)
     (257, 104, 16, 1),     # eight per chunk
