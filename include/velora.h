@@ -37,8 +37,9 @@
  *     their first D columns only.
  *   - N == 0 is a successful no-op (velora_init_v: VELORA_ERR_DEGENERATE_V).
  *   - Vector (128-bit) kernels are used when base pointers are 16-byte aligned,
- *     leading dimensions are multiples of 16 bytes and Dsub is a multiple of 8;
- *     otherwise the element-wise kernels run (same results, lower speed).  The
+ *     leading dimensions are multiples of 16 bytes and Dsub is a multiple of 8
+ *     (fastest for 8 * 2^k) or one of 1, 2, 4; otherwise the element-wise kernels
+ *     run (same results, lower speed).  The
  *     tensor-core GEMMs need 16-byte aligned bf16 rows; other cases run on the
  *     CUDA-core GEMM.
  */
