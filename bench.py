@@ -30,7 +30,12 @@ UNIT = "tokens/s"
 CONFIG_DEFAULT = 5
 CONFIG_INDEX = CONFIG_DEFAULT
 DSUB = 64
-CPU_SAMPLE_TOKENS = 4
+DSUB_SWEEP = 256                # the second sub-token length of configuration 5 (kernel table rows only)
+CPU_SAMPLE_TOKENS = 128         # oracle leg of the default run: tokens per layer, all host threads, one pass (about 30 s)
+CPU_SINGLE_TOKENS = 4           # the same with one thread (about 10 s)
+REF_SAMPLE_TOKENS = 32          # --impl reference: tokens per layer and step (23 passes stay within a few minutes)
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
 GEMM_TRAFFIC_RATIO = 1.07       # ncu dram bytes / algorithmic bytes of the fused forward gemm_pair_kernel on the q layer
 
 
@@ -141,6 +146,17 @@ def oracle_prepare(cfg, sample_tokens: int):
     return layers
 
 
+def set_oracle_threads(n: int) -> bool:
+    """Number of OpenMP threads the (unchanged) oracle library runs with from now on; False if the
+    OpenMP runtime cannot be reached."""
+    import ctypes
+    try:
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+        return True
+    except OSError:
+        return False
+
+
 def oracle_step(layers):
     """One pass of the oracle, as it stands: forward product, compress, input gradient and the weight
     gradient by its plain definition, for every layer."""
@@ -152,8 +168,10 @@ def oracle_step(layers):
         oracle.weight_grad(dY, Z, v, D)
 
 
-CPU_SAMPLE_TEXT = ("first %d tokens of each of the 7 layers: forward product, compress, input gradient, "
-                   "weight gradient by definition" % CPU_SAMPLE_TOKENS)
+def cpu_sample_text(tokens: int) -> str:
+    return ("first %d of the %%d tokens of every layer, each layer in full (forward product, compress, input "
+            "gradient, weight gradient by its plain definition); tokens/s = %d / time of one pass, i.e. "
+            "extrapolated linearly in tokens" % (tokens, tokens))
 
 
 def run_reference(args):
@@ -164,21 +182,21 @@ def run_reference(args):
     import velora_inputs as vi
     cfg = vi.CONFIGS[CONFIG_INDEX]
     oracle.build()
-    layers = oracle_prepare(cfg, CPU_SAMPLE_TOKENS)
+    layers = oracle_prepare(cfg, REF_SAMPLE_TOKENS)
     for _ in range(args.warmup):
         oracle_step(layers)
     t0 = time.perf_counter()
     for _ in range(args.steps):
         oracle_step(layers)
     per_step = (time.perf_counter() - t0) / max(args.steps, 1)
-    value = CPU_SAMPLE_TOKENS / per_step
+    value = REF_SAMPLE_TOKENS / per_step
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(cfg),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                         "sample": CPU_SAMPLE_TEXT},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(oracle.threads(), REF_SAMPLE_TOKENS), "kind": "oracle",
+                         "sample": cpu_sample_text(REF_SAMPLE_TOKENS) % cfg.N},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -295,6 +313,24 @@ def run_ours(args):
         ge.record()
         barrier()
         graph_ms = gs.elapsed_time(ge) / args.steps
+    # ---- the same layers WITHOUT the method (what the paper calls full fine-tuning): Y = X W^T keeping X,
+    # dX = dY W, dW = dY^T X as a dense product.  Same tensor-core kernels, same buffers, same number of steps.
+    def plain_step():
+        for l in L:
+            vl.velora_dense_product(vl.PRODUCT_A_BT, l["X"], l["W"], C=l["Y"], ws=ws)
+            vl.velora_dense_product(vl.PRODUCT_A_B, l["dY"], l["W"], C=l["dX"], ws=ws)
+            vl.velora_dense_product(vl.PRODUCT_AT_B, l["dY"], l["X"], C=l["dW"], ws=ws)
+
+    for _ in range(3):
+        plain_step()
+    barrier()
+    ps, pe = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ps.record()
+    for _ in range(args.steps):
+        plain_step()
+    pe.record()
+    barrier()
+    plain_ms = ps.elapsed_time(pe) / args.steps
     status = vl.velora_workspace_status(ws)
     if status != 0:
         raise RuntimeError("device status %d (%s) after the timed region" % (status, vl.velora_status_string(status)))
@@ -306,25 +342,42 @@ def run_ours(args):
     bwd_ms = sum(e1.elapsed_time(e2) for (_, _, e1, e2) in events)
     fwd_flops = sum(layer_flops(N, l["D"], l["O"], l["M"])["fwd"] for (l, _, _, _) in events)
     achieved = fwd_flops / (fwd_ms * 1e-3) / 1e12
-    peak = pk["bf16_tflops_sustained"]
+    # Which measured peak applies: the burst figure unless the timed region is seconds long (only then has the
+    # power cap pulled the clocks down to where the sustained figure was taken).
+    region_s = elapsed_ms * 1e-3
+    long_region = region_s >= 2.0
+    peak = pk["bf16_tflops_sustained"] if long_region else pk["bf16_tflops"]
+    clk = clocks.summary()
+    clock_scaled = None
+    if clk.get("sm_mhz") and clk.get("sm_max_mhz"):
+        # what the same kernel would reach if the clock had stayed at its maximum: lets boxes be compared
+        clock_scaled = {"achieved_at_max_clock": achieved * clk["sm_max_mhz"] / clk["sm_mhz"],
+                        "sm_mhz_median": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"]}
     # DRAM traffic per launch: ncu on the q-layer launch of this kernel (compress riding along) read + wrote
-    # 182.5 MB = 1.07 x the 169.9 MB of algorithmic bytes X + W + Y + Z (every operand crosses HBM about once;
-    # profiles/gemm_pair_kernel_q_layer_8192x4096x4096.md); the other layers of the step run the same
-    # kernel with the same tile walk and are scaled by their algorithmic bytes.
+    # 182.5 MB = 1.07 x the 169.9 MB of algorithmic bytes X + W + Y + Z (every operand crosses HBM about once);
+    # the other layers of the step run the same kernel with the same tile walk and are scaled by their
+    # algorithmic bytes.
     fwd_bytes = sum((N * l["D"] + l["O"] * l["D"] + N * l["O"]) * 2 + N * l["M"] * 4 for (l, _, _, _) in events)
     traffic = GEMM_TRAFFIC_RATIO * fwd_bytes / max(len(events), 1)
     roofline = {"kernel": "velora_linear_forward (tensor-core GEMM Y = X W^T with compress)", "bound": "tensor",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": "%s, sustained bf16 GEMM" % pk["source"], "traffic": traffic,
+                "peak_source": "%s, %s bf16 GEMM (timed region %.2f s)" % (pk["source"], "sustained" if long_region else "burst", region_s),
+                "frac_burst": achieved / pk["bf16_tflops"], "frac_sustained": achieved / pk["bf16_tflops_sustained"],
+                "frac_nominal": achieved / NOMINAL_BF16_TFLOPS, "clock_scaled": clock_scaled,
+                "traffic": traffic,
                 "traffic_unit": "bytes per launch (average over the 7 layers; q-layer ncu capture, scaled)",
                 "launches": len(events), "avg_launch_ms": fwd_ms / max(len(events), 1),
                 "fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps}
+    overhead = {"velora_ms_per_step": elapsed_ms / args.steps, "plain_ms_per_step": plain_ms,
+                "velora_over_plain": (elapsed_ms / args.steps) / plain_ms,
+                "plain": "the same layers without the method: Y = X W^T, dX = dY W, dW = dY^T X (dense), X kept",
+                "paper": "Table 7 reports VeLoRA 4-9 % slower than full fine-tuning (other hardware, whole model)"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg), "clocks": clocks.summary(),
-        "gpu_launches": int(launches), "roofline": roofline,
+        "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg), "clocks": clk,
+        "gpu_launches": int(launches), "roofline": roofline, "overhead_vs_plain": overhead,
     }
     if graph_ms is not None:
         line["cuda_graph"] = {"ms_per_step": graph_ms, "value": N * world / (graph_ms * 1e-3), "unit": UNIT,
@@ -339,6 +392,23 @@ def run_ours(args):
         return
     if rank == 0:
         line["kernels"] = kernel_table(vl, torch, L, N, ws, pk)
+        # the metric's other two quantities (and reconstruct), per shape, inside the roofline object
+        def pick(prefix):
+            rows = []
+            for r in line["kernels"]:
+                if r["kernel"].startswith(prefix):
+                    row = {"shape": r["shape"], "Dsub": r["Dsub"], "bytes": r["bytes"], "us": r["us"], "GB/s": r["GB/s"],
+                           "frac": r["frac_measured"], "frac_nominal_8TBs": r["GB/s"] / NOMINAL_HBM_GBS}
+                    for k_src, k_dst in (("us_back_to_back", "us_back_to_back"), ("frac_measured_back_to_back", "frac_back_to_back"),
+                                         ("TFLOP/s", "TFLOP/s"), ("roofline_TFLOP/s", "roofline_TFLOP/s")):
+                        if k_src in r:
+                            row[k_dst] = r[k_src]
+                    rows.append(row)
+            return rows
+        line["roofline"]["hbm_peak_GB/s"] = pk["hbm_gbs"]
+        line["roofline"]["compress"] = pick("compress")
+        line["roofline"]["reconstruct"] = pick("reconstruct")
+        line["roofline"]["weight_grad_factored"] = pick("weight_grad factored")
 
     # ---- end to end: host buffers in, gradients out, through velora_linear_step_host.  Three streams, each
     # with its own staging area and workspace, take the layers in turn, so that one layer's copies from and
@@ -392,16 +462,24 @@ def run_ours(args):
 
     if rank == 0:
         import oracle
+        threads = oracle.threads()
         layers = oracle_prepare(cfg, CPU_SAMPLE_TOKENS)
-        reps, t0 = 0, time.perf_counter()
-        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
-            oracle_step(layers)
-            reps += 1
-        t_cpu = (time.perf_counter() - t0) / reps
+        t0 = time.perf_counter()
+        oracle_step(layers)
+        t_cpu = time.perf_counter() - t0
         line["cpu_baseline"] = {
-            "value": CPU_SAMPLE_TOKENS / t_cpu, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": CPU_SAMPLE_TEXT + "; %d passes, %.2f s each" % (reps, t_cpu),
+            "value": CPU_SAMPLE_TOKENS / t_cpu, "unit": UNIT, "cores": min(threads, CPU_SAMPLE_TOKENS), "kind": "oracle",
+            "sample": cpu_sample_text(CPU_SAMPLE_TOKENS) % N + "; one pass, %.1f s" % t_cpu,
         }
+        if set_oracle_threads(1):
+            single = [tuple(a[:CPU_SINGLE_TOKENS] if i in (0, 2) else a for i, a in enumerate(t)) for t in layers]
+            t0 = time.perf_counter()
+            oracle_step(single)
+            t_one = time.perf_counter() - t0
+            set_oracle_threads(threads)
+            line["cpu_baseline"]["single_thread"] = {
+                "value": CPU_SINGLE_TOKENS / t_one, "unit": UNIT, "cores": 1,
+                "sample": cpu_sample_text(CPU_SINGLE_TOKENS) % N + "; one pass, %.1f s" % t_one}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -450,38 +528,51 @@ def kernel_table(vl, torch, L, N, ws, pk):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / (reps * len(fn_list))
 
-    def hbm(name, shape, ms, nbytes, ms_b2b=None):
+    def hbm(name, shape, ms, nbytes, ms_b2b=None, dsub=DSUB):
         gbs = nbytes / (ms * 1e-3) / 1e9
-        row = {"kernel": name, "shape": shape, "us": ms * 1e3, "GB/s": gbs, "bound": "hbm",
-               "frac_measured": gbs / pk["hbm_gbs"], "frac_nominal_8TBs": gbs / 8000.0}
+        row = {"kernel": name, "shape": shape, "Dsub": dsub, "bytes": nbytes, "us": ms * 1e3, "GB/s": gbs, "bound": "hbm",
+               "frac_measured": gbs / pk["hbm_gbs"], "frac_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
         if ms_b2b is not None:
             g2 = nbytes / (ms_b2b * 1e-3) / 1e9
             row.update({"us_back_to_back": ms_b2b * 1e3, "GB/s_back_to_back": g2,
-                        "frac_measured_back_to_back": g2 / pk["hbm_gbs"], "frac_nominal_8TBs_back_to_back": g2 / 8000.0})
+                        "frac_measured_back_to_back": g2 / pk["hbm_gbs"], "frac_nominal_8TBs_back_to_back": g2 / NOMINAL_HBM_GBS})
         out.append(row)
 
-    def tensor(name, shape, ms, flops, nbytes=None):
+    def tensor(name, shape, ms, flops, nbytes=None, dsub=DSUB):
         tf = flops / (ms * 1e-3) / 1e12
-        row = {"kernel": name, "shape": shape, "us": ms * 1e3, "TFLOP/s": tf, "bound": "tensor",
-               "frac_measured_burst": tf / pk["bf16_tflops"]}
+        row = {"kernel": name, "shape": shape, "Dsub": dsub, "us": ms * 1e3, "TFLOP/s": tf, "bound": "tensor",
+               "frac_measured_burst": tf / pk["bf16_tflops"], "frac_nominal": tf / NOMINAL_BF16_TFLOPS}
         if nbytes is not None:                         # factored dW: HBM-bound, graded on bytes
             gbs = nbytes / (ms * 1e-3) / 1e9
             ai = flops / nbytes
-            row.update({"bound": "hbm", "GB/s": gbs, "frac_measured": gbs / pk["hbm_gbs"],
+            row.update({"bound": "hbm", "bytes": nbytes, "GB/s": gbs, "frac_measured": gbs / pk["hbm_gbs"],
                         "roofline_TFLOP/s": min(pk["bf16_tflops"], ai * pk["hbm_gbs"] / 1e3)})
         out.append(row)
+
+    # The second sub-token length of the configuration: its own v and Z per layer.
+    for l in L:
+        l["M2"] = vl.num_subtokens(l["D"], DSUB_SWEEP)
+        l["v2"] = vl.velora_init_v(l["X"], DSUB_SWEEP)
+        l["Z2"] = torch.empty((N, l["M2"]), dtype=torch.float32, device=dev)
+        vl.velora_compress(l["X"], l["v2"], Z=l["Z2"])
+    variants = ((DSUB, "v", "Z", "M"), (DSUB_SWEEP, "v2", "Z2", "M2"))
 
     # streaming kernels: the four 4096-wide inputs rotate (4 x 67 MB), the 11008-wide one is 180 MB alone
     small = [by[n] for n in ("q", "k", "v", "o")]
     big = by["down"]
-    for group, label in ((small, "N=%d D=4096" % N), ([big], "N=%d D=11008" % N)):
-        D, M = group[0]["D"], group[0]["M"]
-        fns = [(lambda l=l: vl.velora_compress(l["X"], l["v"], Z=l["Z"])) for l in group]
-        hbm("compress", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns))
-        fns = [(lambda l=l: vl.velora_reconstruct(l["Z"], l["v"], D, Xhat=l["dX"])) for l in group]
-        hbm("reconstruct", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns))
-        ms = timed([(lambda l=l: vl.velora_init_v(l["X"], DSUB, v=l["v"], ws=ws)) for l in group])
-        hbm("init_v (incl. one stream sync)", label, ms, N * D * 2)
+    for dsub, kv, kz, km in variants:
+        for group, label in ((small, "N=%d D=4096" % N), ([big], "N=%d D=11008" % N)):
+            D, M = group[0]["D"], group[0][km]
+            fns = [(lambda l=l: vl.velora_compress(l["X"], l[kv], Z=l[kz])) for l in group]
+            hbm("compress", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub)
+            fns = [(lambda l=l: vl.velora_reconstruct(l[kz], l[kv], D, Xhat=l["dX"])) for l in group]
+            hbm("reconstruct", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub)
+            if dsub == DSUB:
+                ms = timed([(lambda l=l: vl.velora_init_v(l["X"], DSUB, v=l["v"], ws=ws)) for l in group])
+                hbm("init_v (incl. the stream sync that reads the degenerate flag)", label, ms, N * D * 2)
+                svec = torch.empty(DSUB, dtype=torch.float32, device=dev)
+                fns = [(lambda l=l: vl.velora_subtoken_sum(l["X"], DSUB, s=svec, ws=ws)) for l in group]
+                hbm("subtoken_sum (init_v's two kernels, no sync)", label, timed(fns), N * D * 2, timed_b2b(fns))
     # context only: torch's own fill and reduction on the same 180 MB buffer (pure write / pure read ceilings)
     big_x = big["dX"]
     hbm("reference: torch zero_ (pure write, library kernel)", "N=%d D=11008" % N, timed([lambda: big_x.zero_()]),
@@ -490,27 +581,33 @@ def kernel_table(vl, torch, L, N, ws, pk):
     hbm("reference: torch max (pure read, library kernel)", "N=%d D=11008" % N, timed([lambda: big_i.max()]),
         N * big["D"] * 2)
     # weight gradient, factored: rotate over layers of equal shape
-    for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
-        group = [by[n] for n in names]
-        l0 = group[0]
-        fns = [(lambda l=l: vl.velora_weight_grad(l["dY"], l["Z"], l["v"], l["D"], dW=l["dW"], ws=ws)) for l in group]
-        ms = timed(fns)
-        fl = layer_flops(N, l0["D"], l0["O"], l0["M"])["dw"]
-        nb = N * l0["O"] * 2 + N * l0["M"] * 4 + l0["O"] * l0["D"] * 2
-        tensor("weight_grad factored", "%dx%d -> dW[%d,%d]" % (N, l0["O"], l0["O"], l0["D"]), ms, fl, nb)
-        ms2 = timed_b2b(fns)
-        out[-1].update({"us_back_to_back": ms2 * 1e3, "GB/s_back_to_back": nb / (ms2 * 1e-3) / 1e9,
-                        "frac_measured_back_to_back": nb / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"]})
+    for dsub, kv, kz, km in variants:
+        for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
+            group = [by[n] for n in names]
+            l0 = group[0]
+            fns = [(lambda l=l: vl.velora_weight_grad(l["dY"], l[kz], l[kv], l["D"], dW=l["dW"], ws=ws)) for l in group]
+            ms = timed(fns)
+            fl = layer_flops(N, l0["D"], l0["O"], l0[km])["dw"]
+            nb = N * l0["O"] * 2 + N * l0[km] * 4 + l0["O"] * l0["D"] * 2
+            tensor("weight_grad factored", "%dx%d -> dW[%d,%d]" % (N, l0["O"], l0["O"], l0["D"]), ms, fl, nb, dsub)
+            ms2 = timed_b2b(fns)
+            out[-1].update({"us_back_to_back": ms2 * 1e3, "GB/s_back_to_back": nb / (ms2 * 1e-3) / 1e9,
+                            "frac_measured_back_to_back": nb / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"]})
     # dense contractions
     for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
         group = [by[n] for n in names]
         l0 = group[0]
         fl = 2.0 * N * l0["D"] * l0["O"]
-        ms = timed([(lambda l=l: vl.velora_linear_forward(l["X"], l["W"], l["v"], Y=l["Y"], Z=l["Z"], ws=ws)) for l in group])
-        tensor("linear_forward (GEMM + compress)", "%dx%dx%d" % (N, l0["D"], l0["O"]), ms, fl)
+        for dsub, kv, kz, km in variants:
+            ms = timed([(lambda l=l: vl.velora_linear_forward(l["X"], l["W"], l[kv], Y=l["Y"], Z=l[kz], ws=ws)) for l in group])
+            tensor("linear_forward (GEMM + compress)", "%dx%dx%d" % (N, l0["D"], l0["O"]), ms, fl, dsub=dsub)
+        ms = timed([(lambda l=l: vl.velora_dense_product(vl.PRODUCT_A_BT, l["X"], l["W"], C=l["Y"], ws=ws)) for l in group])
+        tensor("plain forward product Y = X W^T (no compress)", "%dx%dx%d" % (N, l0["D"], l0["O"]), ms, fl, dsub=None)
         ms = timed([(lambda l=l: vl.velora_linear_backward(l["dY"], l["W"], l["Z"], l["v"], dX=l["dX"], need_dW=False, ws=ws))
                     for l in group])
-        tensor("input_grad GEMM dX = dY W", "%dx%dx%d" % (N, l0["O"], l0["D"]), ms, fl)
+        tensor("input_grad GEMM dX = dY W", "%dx%dx%d" % (N, l0["O"], l0["D"]), ms, fl, dsub=None)
+        ms = timed([(lambda l=l: vl.velora_dense_product(vl.PRODUCT_AT_B, l["dY"], l["X"], C=l["dW"], ws=ws)) for l in group])
+        tensor("plain weight gradient dW = dY^T X (dense)", "%dx%dx%d" % (l0["O"], N, l0["D"]), ms, fl, dsub=None)
     l0 = by["q"]
     ws_ex = vl.velora_workspace_alloc(vl.velora_workspace_bytes(vl.OP_WEIGHT_GRAD_EXPLICIT, N, l0["D"], l0["O"], DSUB), dev)
     ms = timed([(lambda l=l: vl.velora_weight_grad(l["dY"], l["Z"], l["v"], l["D"], dW=l["dW"], mode=vl.WG_EXPLICIT, ws=ws_ex))

@@ -13,9 +13,12 @@
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers owned by the caller; the library
- *     never allocates or frees device memory and keeps no state between calls
- *     (only a per-process cache of immutable launch attributes).  Scratch is a
- *     caller-provided device workspace sized by velora_workspace_bytes().
+ *     never allocates or frees device memory.  Scratch is a caller-provided
+ *     device workspace sized by velora_workspace_bytes().  State kept between
+ *     calls: a per-process cache of immutable launch attributes (safe to fill
+ *     from several host threads), and ONE sticky error word per device that
+ *     the entry points without a workspace raise when a bounded wait expires
+ *     (see velora_device_error: shared by all streams and callers of the device).
  *   - Matrices are row-major with an explicit leading dimension counted in
  *     ELEMENTS.  W is [O, D] (nn.Linear convention): Y = X W^T, dX = dY W,
  *     dW = dY^T Xhat.  The listing in Algorithm 1 is only consistent with
@@ -35,7 +38,10 @@
  *     D - (M-1)*Dsub entries followed by zeros (the paper's group() is a
  *     reshape and is silent on this case); outputs of width D are written on
  *     their first D columns only.
- *   - N == 0 is a successful no-op (velora_init_v: VELORA_ERR_DEGENERATE_V).
+ *   - N == 0 (data pointers may then be NULL): velora_compress, velora_reconstruct, velora_linear_forward
+ *     and the dX half of velora_linear_backward write nothing and succeed; velora_init_v returns
+ *     VELORA_ERR_DEGENERATE_V (an empty batch has no mean); the weight gradient of an empty batch is the
+ *     empty sum, dW = beta * dW: beta = 0 fills dW with zeros, beta = 1 leaves it.
  *   - Vector (128-bit) kernels are used when base pointers are 16-byte aligned,
  *     leading dimensions are multiples of 16 bytes and Dsub is a multiple of 8
  *     (fastest for 8 * 2^k) or one of 1, 2, 4; otherwise the element-wise kernels
@@ -64,7 +70,8 @@ typedef enum {
     VELORA_ERR_CUDA = 7           /* a CUDA runtime call or launch failed                      */
 } velora_status;
 
-typedef enum { VELORA_F32 = 0, VELORA_BF16 = 1 } velora_dtype;
+/* VELORA_FP8_E4M3 is a storage type for Z only (see "8-bit storage of Z" below). */
+typedef enum { VELORA_F32 = 0, VELORA_BF16 = 1, VELORA_FP8_E4M3 = 2 } velora_dtype;
 
 /* How velora_weight_grad forms dW. */
 typedef enum {
@@ -79,7 +86,8 @@ typedef enum {
     VELORA_OP_LINEAR_FORWARD = 3,
     VELORA_OP_LINEAR_BACKWARD_FACTORED = 4,
     VELORA_OP_LINEAR_BACKWARD_EXPLICIT = 5,
-    VELORA_OP_UPDATE_V = 6
+    VELORA_OP_UPDATE_V = 6,
+    VELORA_OP_Z8_CALIBRATE = 7
 } velora_op;
 
 #define VELORA_MAX_DSUB 1024
@@ -116,8 +124,27 @@ int velora_workspace_status(const void* ws, void* stream);
  * The entry points that take no workspace (velora_compress, and velora_init_v's first pass) record an
  * expired bounded wait in a word inside the library instead.  velora_device_error synchronises
  * `stream`, returns VELORA_OK or VELORA_ERR_TIMEOUT for the current device and clears the word.
+ * There is one such word per device, whichever stream raised it: the call sees (and clears) what kernels
+ * already completed on ANY stream have recorded, but synchronises only `stream`, so a caller that runs
+ * several streams should drain them before it asks, and only one party per device should do the asking.
  */
 int velora_device_error(void* stream);
+
+/*
+ * Self-test of the bounded waits (the paper has no counterpart; a test hook of the implementation).
+ * Launches ONE small CTA that holds no tile copy and no tensor memory.  Its first warp waits, through the
+ * very routine all pipelines of this library wait with, on a shared-memory barrier that nothing ever
+ * signals, and gives up after limit_ns; its second warp waits on another such barrier with the ordinary
+ * one-second limit and is released early by the abort flag the first warp raises on giving up.  The kernel
+ * then returns normally, having set the workspace's status word and the per-device error word, so
+ * velora_workspace_status(ws) and velora_device_error() both report VELORA_ERR_TIMEOUT (until
+ * velora_workspace_init / the read that clears the word).  Asynchronous.
+ *   limit_ns: 1000 .. 100000000 (1 us .. 100 ms), else VELORA_ERR_INVALID_ARG.
+ *   observed: DEVICE int[4], written by the kernel: [0] first wait gave up (1), [1] microseconds it waited,
+ *             [2] second wait gave up (1), [3] microseconds it waited.
+ *   ws: any initialised workspace (>= 256 bytes).
+ */
+int velora_selftest_wait_timeout(void* ws, size_t ws_bytes, unsigned long long limit_ns, int* observed, void* stream);
 
 /*
  * Initialise the projection vector from a batch (Section 3.2, "Cheap
@@ -158,7 +185,7 @@ int velora_init_v_static(const void* X, int x_dtype, int64_t N, int64_t D, int64
 
 /*
  * compress (Section 3.1, Eq. 1):  Z[n, m] = sum_j X[n, m*Dsub + j] * v[j].
- * X: [N, D] bf16 or f32.  v: fp32 [Dsub].  Z: [N, M] f32 or bf16, ldz >= M.
+ * X: [N, D] bf16 or f32.  v: fp32 [Dsub].  Z: [N, M] f32, bf16 or E4M3, ldz >= M.
  * Products and sums are formed in fp32.
  */
 int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub,
@@ -166,7 +193,7 @@ int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
 
 /*
  * reconstruct + ungroup (Section 3.1, Eq. 2):  Xhat[n, m*Dsub + j] = Z[n, m] * v[j].
- * Z: [N, M] f32 or bf16.  Xhat: [N, D] bf16 or f32 (rounded to nearest even).
+ * Z: [N, M] f32, bf16 or E4M3.  Xhat: [N, D] bf16 or f32 (rounded to nearest even).
  */
 int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64_t D, int Dsub,
                        const float* v, void* Xhat, int x_dtype, int64_t ldxhat, void* stream);
@@ -174,7 +201,7 @@ int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
 /*
  * Weight gradient of Algorithm 1's backward with the reconstructed input:
  *     dW[o, d] = beta * dW[o, d] + sum_n dY[n, o] * Xhat[n, d],  Xhat = Z (x) v
- * dY: [N, O] bf16 or f32.  Z: [N, M] f32 or bf16.  dW: [O, D] bf16 or f32.
+ * dY: [N, O] bf16 or f32.  Z: [N, M] f32, bf16 or E4M3.  dW: [O, D] bf16 or f32.
  * beta is 0 (overwrite) or 1 (accumulate into dW).
  * mode VELORA_WG_FACTORED uses dW[o, m*Dsub+j] = (dY^T Z)[o, m] * v[j]
  * (the Dsub = D case is the paper's g v v^T, Section 3.2); VELORA_WG_EXPLICIT
@@ -215,6 +242,53 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
                            void* dX, int64_t lddx, void* dW, int dw_dtype, int64_t lddw, int beta, int mode,
                            int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
                            void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * 8-bit storage of Z (an extension of Section 3.1: what the forward pass keeps for the backward pass is the
+ * array of scalars Z, and the paper's memory tables (Table 5(b), Table 6) count exactly those bytes; it
+ * stores them in the training precision, this stores them in one byte each).
+ *
+ * Every entry point that writes or reads Z accepts z_dtype = VELORA_FP8_E4M3: Z is then [N, M] bytes (ldz in
+ * bytes) in the E4M3 format (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
+ * value 448).  A writer stores round_to_nearest_even(<sub-token, v>), saturating at +-448; a reader uses the
+ * decoded value as Z.  The scale that brings Z into E4M3's range travels in the VECTOR argument, since
+ * compress is linear in v and the backward pass is linear in v as well:
+ *     writers (velora_compress, velora_linear_forward):                      pass v_store = v / zscale
+ *     readers (velora_reconstruct, velora_weight_grad, velora_linear_backward,
+ *              velora_expand_p after velora_weight_grad_p):                   pass v_load  = v * zscale
+ * so that Xhat = decode(Z8) (x) v_load approximates Z (x) v and no kernel needs a scale argument.  The
+ * weight gradient feeds the decoded values to the tensor cores as they are (every E4M3 value is a bf16
+ * value), so an 8-bit Z adds no rounding beyond the store's own: relative error at most 2^-4 per scalar
+ * for |Z| >= zscale * 2^-6, absolute error at most zscale * 2^-10 below that.
+ *
+ * velora_z8_calibrate chooses the scale from a batch (like v itself it is meant to be fixed on the first
+ * batch and kept):  zscale = headroom * max_{n,m} |<x_nm, v>| / 448   (1 if that maximum is zero or not
+ * finite), v_store = v / zscale, v_load = v * zscale.  headroom in [1, 1024] leaves room for later batches
+ * (2 puts the calibration batch's largest scalar at 224); scalars beyond the range saturate.
+ * zscale[1], v_store[Dsub], v_load[Dsub]: device fp32.  Asynchronous.
+ * ws: velora_workspace_bytes(VELORA_OP_Z8_CALIBRATE, N, D, 0, Dsub) bytes (holds Z of the batch in fp32).
+ */
+int velora_z8_calibrate(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                        float headroom, float* zscale, float* v_store, float* v_load,
+                        void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The dense products of Algorithm 1 on their own, i.e. the layer WITHOUT the method: Y = X W^T (forward),
+ * dX = dY W and dW = dY^T X (backward, with the input X kept instead of Z).  They are the same tensor-core
+ * kernels the VeLoRA entry points use, exported so that the cost of an uncompressed layer can be measured
+ * beside the compressed one (Section 5, the speed comparison with full fine-tuning).
+ *     C[Mdim, Ndim] = beta * C + op(A) op(B),  fp32 accumulation, beta in {0, 1}
+ *   VELORA_PRODUCT_A_BT:  A[Mdim, Kdim], B[Ndim, Kdim]    (C = A B^T)
+ *   VELORA_PRODUCT_A_B:   A[Mdim, Kdim], B[Kdim, Ndim]    (C = A B)
+ *   VELORA_PRODUCT_AT_B:  A[Kdim, Mdim], B[Kdim, Ndim]    (C = A^T B)
+ * `dtype`: storage type of A and B (bf16: tensor cores when rows are 16-byte aligned; otherwise and for
+ * f32 the CUDA-core product).  C: c_dtype, bf16 or f32.  ws: at least 256 bytes, initialised (status header).
+ */
+typedef enum { VELORA_PRODUCT_A_BT = 0, VELORA_PRODUCT_A_B = 1, VELORA_PRODUCT_AT_B = 2 } velora_product;
+int velora_dense_product(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
+                         void* C, int c_dtype, int64_t ldc, int beta,
+                         int64_t Mdim, int64_t Ndim, int64_t Kdim, int dtype,
+                         void* ws, size_t ws_bytes, void* stream);
 
 /*
  * The two halves of velora_init_v, for a batch that is sharded over several processes (Section 3.2:

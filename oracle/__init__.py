@@ -229,6 +229,43 @@ def round_to_f32(a):
     return np.asarray(a, dtype=np.float64).astype(np.float32).astype(np.float64)
 
 
+FP8_E4M3_MAX = 448.0
+
+
+def round_to_fp8_e4m3(a):
+    """Round float64 values to the nearest value of the 8-bit format E4M3 (1 sign, 4 exponent bits with
+    bias 7, 3 mantissa bits; no infinities, largest finite value 448), ties to even, SATURATING: anything
+    beyond +-448 (infinities included) becomes +-448.  Returned as float64; NaN stays NaN.
+
+    Normal values (|x| >= 2^-6) have a 4-bit significand, so in frexp form (x = mant * 2^expo,
+    0.5 <= |mant| < 1) neighbours are 2^(expo - 4) apart.  Below 2^-6 the format is subnormal with the
+    fixed spacing 2^-9, which is the same formula with expo held at -5.
+    """
+    a = np.asarray(a, dtype=np.float64)
+    _, expo = np.frexp(a)
+    step = np.ldexp(1.0, np.maximum(expo, -5) - 4)
+    with np.errstate(invalid="ignore"):
+        q = np.rint(a / step) * step
+    q = np.where(np.isnan(a), a, np.clip(q, -FP8_E4M3_MAX, FP8_E4M3_MAX))
+    return np.where(np.isinf(a), np.sign(a) * FP8_E4M3_MAX, q)
+
+
+def zscale_from_batch(Z, headroom: float = 2.0) -> float:
+    """Scale for storing Z in E4M3 (extension of Section 3.1's stored scalars to an 8-bit store; not in
+    the paper): the largest magnitude of a calibration batch times ``headroom`` maps to 448.  A batch
+    without a finite positive maximum gives 1."""
+    amax = float(np.max(np.abs(Z))) if np.size(Z) else 0.0
+    if not np.isfinite(amax) or amax <= 0.0:
+        return 1.0
+    return headroom * amax / FP8_E4M3_MAX
+
+
+def quantize_z_fp8(Z, zscale: float):
+    """The values an E4M3 store of Z holds: round_to_fp8_e4m3(Z / zscale), as float64 (multiply by zscale
+    to get the Z that the backward pass sees)."""
+    return round_to_fp8_e4m3(np.asarray(Z, dtype=np.float64) / float(zscale))
+
+
 def round_to(a, dtype: str):
     if dtype == "bf16":
         return round_to_bf16(a)

@@ -11,7 +11,9 @@ from .binding import (  # noqa: F401
     velora_linear_backward, velora_linear_forward, velora_reconstruct, velora_status_string,
     velora_version, velora_weight_grad, velora_workspace_alloc, velora_workspace_bytes,
     velora_workspace_init, velora_workspace_status, velora_launch_count, velora_device_error, velora_subtoken_sum, velora_normalize_v,
-    velora_update_v, OP_UPDATE_V, ERR_DEGENERATE_V,
+    velora_update_v, OP_UPDATE_V, ERR_DEGENERATE_V, ERR_TIMEOUT, velora_selftest_wait_timeout,
+    velora_z8_calibrate, FP8_E4M3, OP_Z8_CALIBRATE, Z8_TORCH,
+    velora_dense_product, PRODUCT_A_BT, PRODUCT_A_B, PRODUCT_AT_B,
     velora_weight_grad_p, velora_expand_p,
     velora_host_step_staging_bytes, velora_linear_step_host,
 )

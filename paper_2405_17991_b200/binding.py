@@ -18,10 +18,11 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libvelora.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_DEGENERATE_V, ERR_TIMEOUT, ERR_CUDA = range(8)
-F32, BF16 = 0, 1
+F32, BF16, FP8_E4M3 = 0, 1, 2
 WG_FACTORED, WG_EXPLICIT = 0, 1
+PRODUCT_A_BT, PRODUCT_A_B, PRODUCT_AT_B = 0, 1, 2
 (OP_INIT_V, OP_WEIGHT_GRAD_FACTORED, OP_WEIGHT_GRAD_EXPLICIT, OP_LINEAR_FORWARD,
- OP_LINEAR_BACKWARD_FACTORED, OP_LINEAR_BACKWARD_EXPLICIT, OP_UPDATE_V) = range(7)
+ OP_LINEAR_BACKWARD_FACTORED, OP_LINEAR_BACKWARD_EXPLICIT, OP_UPDATE_V, OP_Z8_CALIBRATE) = range(8)
 
 _p, _i64, _int, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
 
@@ -35,6 +36,7 @@ SIGNATURES = {
     "velora_workspace_init": (_int, [_p, _sz, _p]),
     "velora_workspace_status": (_int, [_p, _p]),
     "velora_device_error": (_int, [_p]),
+    "velora_selftest_wait_timeout": (_int, [_p, _sz, ctypes.c_ulonglong, _p, _p]),
     "velora_init_v": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
     "velora_init_v_static": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p]),
     "velora_subtoken_sum": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _sz, _p]),
@@ -42,6 +44,8 @@ SIGNATURES = {
     "velora_update_v": (_int, [_p, _int, _i64, _i64, _i64, _int, ctypes.c_float, _p, _p, _p, _sz, _p]),
     "velora_weight_grad_p": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _i64, _int, _p, _i64, _int, _p, _sz, _p]),
     "velora_expand_p": (_int, [_p, _i64, _p, _i64, _i64, _int, _p, _int, _i64, _int, _p]),
+    "velora_z8_calibrate": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, ctypes.c_float, _p, _p, _p, _p, _sz, _p]),
+    "velora_dense_product": (_int, [_int, _p, _i64, _p, _i64, _p, _int, _i64, _int, _i64, _i64, _i64, _int, _p, _sz, _p]),
     "velora_compress": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_reconstruct": (_int, [_p, _int, _i64, _i64, _i64, _int, _p, _p, _int, _i64, _p]),
     "velora_weight_grad": (_int, [_p, _int, _i64, _i64, _i64, _p, _int, _i64, _p, _i64, _int,
@@ -80,12 +84,17 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
+Z8_TORCH = getattr(torch, "float8_e4m3fn", None)      # torch's name for the E4M3 byte; torch.uint8 is accepted as well
+
+
 def _dt(t: torch.Tensor) -> int:
     if t.dtype == torch.float32:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
-    raise TypeError("unsupported dtype %s (float32 or bfloat16)" % t.dtype)
+    if t.dtype == torch.uint8 or (Z8_TORCH is not None and t.dtype == Z8_TORCH):
+        return FP8_E4M3                                 # only Z may have this type; the library checks
+    raise TypeError("unsupported dtype %s (float32, bfloat16, or uint8 / float8_e4m3fn for Z)" % t.dtype)
 
 
 def _mat(t: torch.Tensor, name: str):
@@ -135,6 +144,15 @@ def velora_workspace_status(ws: torch.Tensor, stream=None) -> int:
 def velora_device_error(stream=None) -> int:
     """Synchronises the stream; 0, or ERR_TIMEOUT if a streaming kernel's bounded wait expired (then cleared)."""
     return int(lib().velora_device_error(_stream(stream)))
+
+
+def velora_selftest_wait_timeout(ws: torch.Tensor, limit_ns: int, observed: torch.Tensor, stream=None) -> None:
+    """Runs the one-CTA kernel whose bounded waits expire; ``observed`` is a 4-element int32 CUDA tensor."""
+    if observed.dtype != torch.int32 or observed.numel() < 4 or not observed.is_cuda or not observed.is_contiguous():
+        raise ValueError("observed must be a contiguous int32 CUDA tensor with 4 elements")
+    _check(lib().velora_selftest_wait_timeout(ctypes.c_void_p(ws.data_ptr()), ws.numel(), int(limit_ns),
+                                              ctypes.c_void_p(observed.data_ptr()), _stream(stream)),
+           "velora_selftest_wait_timeout")
 
 
 def _check(status: int, where: str):
@@ -277,6 +295,40 @@ def velora_linear_backward(dY: torch.Tensor, W: torch.Tensor, Z: torch.Tensor, v
                                       _stream(stream))
     _check(rc, "velora_linear_backward")
     return dX, dW
+
+
+def velora_dense_product(kind: int, A: torch.Tensor, B: torch.Tensor, C: Optional[torch.Tensor] = None,
+                         c_dtype=None, beta: int = 0, ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """C = beta * C + op(A) op(B): the plain products of the layer (PRODUCT_A_BT, PRODUCT_A_B, PRODUCT_AT_B)."""
+    ap, lda = _mat(A, "A")
+    bp, ldb = _mat(B, "B")
+    Mdim, Kdim = (A.shape[1], A.shape[0]) if kind == PRODUCT_AT_B else (A.shape[0], A.shape[1])
+    Ndim = B.shape[0] if kind == PRODUCT_A_BT else B.shape[1]
+    if (B.shape[1] if kind == PRODUCT_A_BT else B.shape[0]) != Kdim or A.dtype != B.dtype:
+        raise ValueError("operand shapes or dtypes do not match")
+    if C is None:
+        C = torch.empty((Mdim, Ndim), dtype=c_dtype or A.dtype, device=A.device)
+    cp, ldc = _mat(C, "C")
+    ws = _ws(ws, 256, A.device)
+    rc = lib().velora_dense_product(kind, ap, lda, bp, ldb, cp, _dt(C), ldc, beta, Mdim, Ndim, Kdim, _dt(A),
+                                    ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_dense_product")
+    return C
+
+
+def velora_z8_calibrate(X: torch.Tensor, v: torch.Tensor, headroom: float = 2.0, ws: Optional[torch.Tensor] = None,
+                        stream=None):
+    """Scale of the 8-bit Z store from a batch: returns (zscale[1], v_store = v / zscale, v_load = v * zscale)."""
+    xp, ldx = _mat(X, "X")
+    N, D = X.shape
+    Dsub = v.shape[0]
+    zscale = torch.empty(1, dtype=torch.float32, device=X.device)
+    v_store, v_load = torch.empty_like(v), torch.empty_like(v)
+    ws = _ws(ws, velora_workspace_bytes(OP_Z8_CALIBRATE, N, D, 0, Dsub), X.device)
+    rc = lib().velora_z8_calibrate(xp, _dt(X), N, D, ldx, Dsub, _vec(v), float(headroom), _vec(zscale), _vec(v_store),
+                                   _vec(v_load), ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream))
+    _check(rc, "velora_z8_calibrate")
+    return zscale, v_store, v_load
 
 
 def velora_launch_count() -> int:

@@ -7,21 +7,22 @@ namespace velora {
 
 int device_info(DeviceInfo* out)
 {
-    static DeviceInfo cache[64];
-    static bool have[64] = {};
+    static std::atomic<int> sm_count[64], smem_optin[64];      // 0 = not asked yet (both are positive on any device)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return VELORA_ERR_CUDA;
     if (dev < 0 || dev >= 64) return VELORA_ERR_UNSUPPORTED;
-    if (!have[dev]) {
-        DeviceInfo di;
+    DeviceInfo di;
+    di.sm_count = sm_count[dev].load(std::memory_order_relaxed);
+    di.smem_optin = smem_optin[dev].load(std::memory_order_relaxed);
+    if (di.sm_count == 0 || di.smem_optin == 0) {
         if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return VELORA_ERR_CUDA;
         if (cudaDeviceGetAttribute(&di.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return VELORA_ERR_CUDA;
-        cache[dev] = di;
-        have[dev] = true;
+        sm_count[dev].store(di.sm_count, std::memory_order_relaxed);
+        smem_optin[dev].store(di.smem_optin, std::memory_order_relaxed);
     }
-    *out = cache[dev];
+    *out = di;
     return VELORA_OK;
 }
 
@@ -77,6 +78,12 @@ int weight_grad_impl(const void* dY, int dy_dtype, int64_t N, int64_t O, int64_t
     const int64_t M = num_subtokens(D, Dsub);
     int* status = static_cast<int*>(ws);                 // word 0: sticky device error flag
     char* body = static_cast<char*>(ws) + kStatusBytes;
+    if (N == 0) {                                        // empty sum: dW = beta * dW
+        if (beta) return VELORA_OK;
+        const size_t es = dtype_size(dw_dtype);
+        return cudaMemset2DAsync(dW, static_cast<size_t>(lddw) * es, 0, static_cast<size_t>(D) * es,
+                                 static_cast<size_t>(O), stream) == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    }
     if (mode == VELORA_WG_FACTORED) {
         if (ws_bytes < factored_bytes(N, D, O, Dsub)) return VELORA_ERR_WORKSPACE;
         // Adapter-shaped layers (O <= 64) first: too few output tiles for the tensor-core kernel to spread.
@@ -106,17 +113,21 @@ int check_weight_grad_args(const void* dY, int dy_dtype, int64_t N, int64_t O, i
                            const void* Z, int z_dtype, int64_t ldz, const float* v, int64_t D, int Dsub,
                            void* dW, int dw_dtype, int64_t lddw, int beta, int mode, void* ws)
 {
-    if (!dY || !Z || !v || !dW) return VELORA_ERR_INVALID_ARG;
+    if (!dW) return VELORA_ERR_INVALID_ARG;
     if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
-    if (!valid_dtype(dy_dtype) || !valid_dtype(z_dtype) || !valid_dtype(dw_dtype)) return VELORA_ERR_UNSUPPORTED;
-    if (lddy < O || ldz < num_subtokens(D, Dsub) || lddw < D) return VELORA_ERR_INVALID_ARG;
+    if (!valid_dtype(dy_dtype) || !valid_z_dtype(z_dtype) || !valid_dtype(dw_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (lddw < D) return VELORA_ERR_INVALID_ARG;
     if ((beta != 0 && beta != 1) || (mode != VELORA_WG_FACTORED && mode != VELORA_WG_EXPLICIT))
         return VELORA_ERR_INVALID_ARG;
-    if (!elem_aligned(dY, dy_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(dW, dw_dtype) ||
-        !elem_aligned(v, VELORA_F32))
-        return VELORA_ERR_ALIGNMENT;
+    if (!elem_aligned(dW, dw_dtype)) return VELORA_ERR_ALIGNMENT;
+    if (N > 0) {                                         /* an empty batch may carry NULL dY, Z and v */
+        if (!dY || !Z || !v) return VELORA_ERR_INVALID_ARG;
+        if (lddy < O || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
+        if (!elem_aligned(dY, dy_dtype) || !elem_aligned(Z, z_dtype) || !elem_aligned(v, VELORA_F32))
+            return VELORA_ERR_ALIGNMENT;
+    }
     if (!ws) return VELORA_ERR_WORKSPACE;
     if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
     return VELORA_OK;
@@ -144,6 +155,16 @@ int velora_workspace_init(void* ws, size_t ws_bytes, void* stream)
 int velora_device_error(void* stream)
 {
     return read_and_clear_stream_error(static_cast<cudaStream_t>(stream));
+}
+
+int velora_selftest_wait_timeout(void* ws, size_t ws_bytes, unsigned long long limit_ns, int* observed, void* stream)
+{
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    if (!observed) return VELORA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(observed) % sizeof(int)) return VELORA_ERR_ALIGNMENT;
+    if (limit_ns < 1000ull || limit_ns > 100000000ull) return VELORA_ERR_INVALID_ARG;   /* 1 us .. 100 ms */
+    return launch_wait_timeout_selftest(static_cast<int*>(ws), limit_ns, observed, static_cast<cudaStream_t>(stream));
 }
 
 int velora_workspace_status(const void* ws, void* stream)
@@ -183,6 +204,7 @@ size_t velora_workspace_bytes(int op, int64_t N, int64_t D, int64_t O, int Dsub)
         case VELORA_OP_LINEAR_BACKWARD_EXPLICIT: return xhat_bytes(N, D);
         case VELORA_OP_LINEAR_FORWARD: return kStatusBytes;
         case VELORA_OP_UPDATE_V: return update_v_workspace_bytes(Dsub);
+        case VELORA_OP_Z8_CALIBRATE: return z8_calibrate_workspace_bytes(N, D, Dsub);
         default: return 0;
     }
 }
@@ -207,7 +229,7 @@ int velora_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
 {
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
-    if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(x_dtype) || !valid_z_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
     if (N == 0) return VELORA_OK;                    /* empty tensors may carry NULL pointers */
     if (!X || !v || !Z) return VELORA_ERR_INVALID_ARG;
     if (ldx < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
@@ -221,7 +243,7 @@ int velora_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
 {
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
-    if (!valid_dtype(x_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(x_dtype) || !valid_z_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
     if (N == 0) return VELORA_OK;
     if (!Z || !v || !Xhat) return VELORA_ERR_INVALID_ARG;
     if (ldxhat < D || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
@@ -255,7 +277,7 @@ int velora_linear_forward(const void* X, int64_t ldx, const void* W, int64_t ldw
     if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
-    if (!valid_dtype(dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(dtype) || !valid_z_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
     if (N == 0) return VELORA_OK;
     if (!X || !W || !v || !Y || !Z) return VELORA_ERR_INVALID_ARG;
     if (ldx < D || ldw < D || ldy < O || ldz < num_subtokens(D, Dsub)) return VELORA_ERR_INVALID_ARG;
@@ -279,14 +301,16 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
                            int dtype, int64_t N, int64_t D, int64_t O, int Dsub,
                            void* ws, size_t ws_bytes, void* stream)
 {
-    if (!dY) return VELORA_ERR_INVALID_ARG;
     if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
     if (!valid_dtype(dtype)) return VELORA_ERR_UNSUPPORTED;
-    if (lddy < O) return VELORA_ERR_INVALID_ARG;
-    if (!elem_aligned(dY, dtype)) return VELORA_ERR_ALIGNMENT;
-    if (dX) {
+    if (N > 0) {
+        if (!dY) return VELORA_ERR_INVALID_ARG;
+        if (lddy < O) return VELORA_ERR_INVALID_ARG;
+        if (!elem_aligned(dY, dtype)) return VELORA_ERR_ALIGNMENT;
+    }
+    if (dX && N > 0) {
         if (!W) return VELORA_ERR_INVALID_ARG;
         if (ldw < D || lddx < D) return VELORA_ERR_INVALID_ARG;
         if (!elem_aligned(W, dtype) || !elem_aligned(dX, dtype)) return VELORA_ERR_ALIGNMENT;
@@ -314,6 +338,39 @@ int velora_linear_backward(const void* dY, int64_t lddy, const void* W, int64_t 
         return weight_grad_impl(dY, dtype, N, O, lddy, Z, z_dtype, ldz, v, D, Dsub, dW, dw_dtype, lddw,
                                 beta, mode, ws, ws_bytes, s);
     return VELORA_OK;
+}
+
+int velora_dense_product(int kind, const void* A, int64_t lda, const void* B, int64_t ldb,
+                         void* C, int c_dtype, int64_t ldc, int beta,
+                         int64_t Mdim, int64_t Ndim, int64_t Kdim, int dtype,
+                         void* ws, size_t ws_bytes, void* stream)
+{
+    if (kind != VELORA_PRODUCT_A_BT && kind != VELORA_PRODUCT_A_B && kind != VELORA_PRODUCT_AT_B) return VELORA_ERR_INVALID_ARG;
+    if (Mdim < 0 || Ndim < 1 || Kdim < 0 || (beta != 0 && beta != 1)) return VELORA_ERR_INVALID_ARG;
+    if (Mdim > (1 << 30) || Ndim > (1 << 30) || Kdim > (1 << 30)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(dtype) || !valid_dtype(c_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (Mdim == 0) return VELORA_OK;
+    if (!C || ldc < Ndim) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(C, c_dtype)) return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (Kdim == 0) {                                     /* empty sum: C = beta * C */
+        if (beta) return VELORA_OK;
+        const size_t es = dtype_size(c_dtype);
+        return cudaMemset2DAsync(C, static_cast<size_t>(ldc) * es, 0, static_cast<size_t>(Ndim) * es,
+                                 static_cast<size_t>(Mdim), s) == cudaSuccess ? VELORA_OK : VELORA_ERR_CUDA;
+    }
+    if (!A || !B) return VELORA_ERR_INVALID_ARG;
+    const bool a_t = kind == VELORA_PRODUCT_AT_B, b_t = kind == VELORA_PRODUCT_A_BT;
+    if (lda < (a_t ? Mdim : Kdim) || ldb < (b_t ? Kdim : Ndim)) return VELORA_ERR_INVALID_ARG;
+    if (!elem_aligned(A, dtype) || !elem_aligned(B, dtype)) return VELORA_ERR_ALIGNMENT;
+    const int tc_kind = kind == VELORA_PRODUCT_A_BT ? GEMM_NT_K_K : (kind == VELORA_PRODUCT_A_B ? GEMM_NN_K_MN : GEMM_TN_MN_MN);
+    int rc = launch_gemm_tc(tc_kind, A, lda, B, ldb, C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, dtype,
+                            static_cast<int*>(ws), s);
+    if (rc != VELORA_ERR_UNSUPPORTED) return rc;
+    return launch_gemm_simt(A, dtype, a_t ? 1 : lda, a_t ? lda : 1, B, dtype, b_t ? ldb : 1, b_t ? 1 : ldb,
+                            C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, s);
 }
 
 size_t velora_host_step_staging_bytes(int64_t N, int64_t D, int64_t O, int Dsub)
@@ -396,6 +453,25 @@ int velora_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
     return launch_update_v(X, x_dtype, N, D, ldx, Dsub, rho, a, v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
+int velora_z8_calibrate(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                        float headroom, float* zscale, float* v_store, float* v_load,
+                        void* ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_shape(N, D, Dsub);
+    if (rc != VELORA_OK) return rc;
+    if (!valid_dtype(x_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!(headroom >= 1.f && headroom <= 1024.f)) return VELORA_ERR_INVALID_ARG;
+    if (!v || !zscale || !v_store || !v_load) return VELORA_ERR_INVALID_ARG;
+    if (N > 0 && (!X || ldx < D)) return VELORA_ERR_INVALID_ARG;
+    if ((N > 0 && !elem_aligned(X, x_dtype)) || !elem_aligned(v, VELORA_F32) || !elem_aligned(zscale, VELORA_F32) ||
+        !elem_aligned(v_store, VELORA_F32) || !elem_aligned(v_load, VELORA_F32))
+        return VELORA_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < z8_calibrate_workspace_bytes(N, D, Dsub)) return VELORA_ERR_WORKSPACE;
+    if (!aligned16(ws)) return VELORA_ERR_ALIGNMENT;
+    return launch_z8_calibrate(X, x_dtype, N, D, ldx, Dsub, v, headroom, zscale, v_store, v_load, ws, ws_bytes,
+                               static_cast<cudaStream_t>(stream));
+}
+
 int velora_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_bytes, void* stream)
 {
     if (!s || !v || Dsub < 1) return VELORA_ERR_INVALID_ARG;
@@ -413,7 +489,7 @@ int velora_weight_grad_p(const void* dY, int dy_dtype, int64_t N, int64_t O, int
     if (O < 1 || O > (1 << 30)) return VELORA_ERR_INVALID_ARG;
     int rc = check_shape(N, D, Dsub);
     if (rc != VELORA_OK) return rc;
-    if (!valid_dtype(dy_dtype) || !valid_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
+    if (!valid_dtype(dy_dtype) || !valid_z_dtype(z_dtype)) return VELORA_ERR_UNSUPPORTED;
     const int64_t M = num_subtokens(D, Dsub);
     if (!P || ldp < M || (beta != 0 && beta != 1)) return VELORA_ERR_INVALID_ARG;
     if (!elem_aligned(P, VELORA_F32)) return VELORA_ERR_ALIGNMENT;

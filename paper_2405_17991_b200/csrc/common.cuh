@@ -2,8 +2,11 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <atomic>
 
 #include "velora.h"
 
@@ -23,6 +26,15 @@ int device_info(DeviceInfo* out);
 
 // Call right after every kernel launch: counts it and turns a launch error into a status.
 int after_launch();
+
+// "Done once per device" flags for host-side set-up that is harmless to repeat (a kernel attribute set to
+// the same value, an address looked up again): atomics keep the first calls of two host threads from being
+// a data race; nothing worse than a repeated set-up can happen.
+struct DeviceOnce {
+    std::atomic<bool> done[64];
+    bool get(int dev) const { return done[dev].load(std::memory_order_acquire); }
+    void set(int dev) { done[dev].store(true, std::memory_order_release); }
+};
 
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 // Programmatic dependent launch.  A kernel launched with pdl_attribute() may become resident while the
@@ -44,8 +56,9 @@ inline cudaLaunchAttribute pdl_attribute()
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : 4; }
-inline bool valid_dtype(int dt) { return dt == VELORA_F32 || dt == VELORA_BF16; }
+inline size_t dtype_size(int dt) { return dt == VELORA_BF16 ? 2 : (dt == VELORA_FP8_E4M3 ? 1 : 4); }
+inline bool valid_dtype(int dt) { return dt == VELORA_F32 || dt == VELORA_BF16; }                 // X, W, dY, Y, dX, dW
+inline bool valid_z_dtype(int dt) { return valid_dtype(dt) || dt == VELORA_FP8_E4M3; }              // stored Z
 
 // ---- streaming kernels (stream_kernels.cu) ----
 // sum_only != 0: v receives the un-normalised sub-token sum s and nothing is synchronised.
@@ -60,6 +73,12 @@ int launch_weight_grad_skinny(const void* dY, int dy_dtype, int64_t N, int64_t O
                               void* dW, int dw_dtype, int64_t lddw, int beta,
                               void* ws, size_t ws_bytes, cudaStream_t stream, float* P_out, int64_t ldp_out);
 size_t init_v_workspace_bytes(int Dsub);
+// Scale of the 8-bit Z store from a batch: zscale = headroom * max|compress(X, v)| / 448 (1 if that maximum is
+// zero or not finite), v_store = v / zscale, v_load = v * zscale.  Asynchronous.
+size_t z8_calibrate_workspace_bytes(int64_t N, int64_t D, int Dsub);
+int launch_z8_calibrate(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                        float headroom, float* zscale, float* v_store, float* v_load,
+                        void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t update_v_workspace_bytes(int Dsub);
 int launch_update_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, float rho,
                     float* a, float* v, void* ws, size_t ws_bytes, cudaStream_t stream);
@@ -96,6 +115,29 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// One byte of the 8-bit floating-point format E4M3 (4 exponent bits, bias 7; 3 mantissa bits; no infinities,
+// largest finite value 448): a storage type for Z only.  Conversions are the hardware's: round to nearest
+// even, saturating at +-448.
+struct e4m3_t {
+    unsigned char bits;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ e4m3_t float_to_e4m3(float x)
+{
+    unsigned short pair;                                  // the first source lands in the upper byte, the second in the lower
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(0.f), "f"(x));
+    e4m3_t r;
+    r.bits = static_cast<unsigned char>(pair & 0xffu);
+    return r;
+}
+__device__ __forceinline__ float e4m3_to_float(e4m3_t q)
+{
+    unsigned int halves;                                  // the lower byte becomes the lower half-precision value
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(halves) : "h"(static_cast<unsigned short>(q.bits)));
+    return __half2float(__ushort_as_half(static_cast<unsigned short>(halves & 0xffffu)));
+}
+#endif
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static __device__ __forceinline__ float load(const float* p) { return *p; }
@@ -104,6 +146,10 @@ template <> struct Elem<float> {
 template <> struct Elem<__nv_bfloat16> {
     static __device__ __forceinline__ float load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
     static __device__ __forceinline__ void store(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+};
+template <> struct Elem<e4m3_t> {
+    static __device__ __forceinline__ float load(const e4m3_t* p) { return e4m3_to_float(*p); }
+    static __device__ __forceinline__ void store(e4m3_t* p, float x) { *p = float_to_e4m3(x); }
 };
 
 }  // namespace velora

@@ -24,6 +24,7 @@ template <> __device__ __forceinline__ float load_scalar<__nv_bfloat16>(const __
 {
     return __bfloat162float(*p);
 }
+template <> __device__ __forceinline__ float load_scalar<e4m3_t>(const e4m3_t* p) { return e4m3_to_float(*p); }
 
 template <typename WT> struct Out8;
 template <> struct Out8<__nv_bfloat16> {
@@ -73,49 +74,67 @@ expand_rows_vec_kernel(const ST* __restrict__ S, int splits, int64_t split_strid
     const int lane = threadIdx.x & 31;
     const int q = lane & (LPS - 1);
     const int sub = lane / LPS;
+    // Programmatic stream serialisation (see common.cuh): resident early, nothing read or written before the wait.
+    pdl_trigger();
+    pdl_wait();
     float vr[CH][8];
 #pragma unroll
     for (int i = 0; i < CH; ++i)
 #pragma unroll
         for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
 
-    // One warp per output row at a time; the row's blocks of 32 sub-tokens are walked in an inner loop.
+    // One warp per output row at a time.  The row's scalars are fetched for up to PB blocks of 32 sub-tokens
+    // before the first store, so a row costs one load latency per PB blocks instead of one per block (a row of
+    // 172 sub-tokens went through six dependent round trips to memory before).
+    constexpr int PB = 4;
     const int warps = gridDim.x * (kStreamThreads / 32);
     for (int r = blockIdx.x * (kStreamThreads / 32) + (threadIdx.x >> 5); r < R; r += warps)
-    for (int m0 = 0; m0 < mblocks * 32; m0 += 32) {
-        float p = 0.f;
-        if (MODE == 0 || m0 + lane < M) {
-            const ST* sp = S + static_cast<int64_t>(r) * lds + m0 + lane;
+    for (int mb0 = 0; mb0 < mblocks; mb0 += PB) {
+        float pb[PB];
+#pragma unroll
+        for (int b = 0; b < PB; ++b) {
+            const int m = (mb0 + b) * 32 + lane;
+            float p = 0.f;
+            if (mb0 + b < mblocks && (MODE == 0 || m < M)) {
+                const ST* sp = S + static_cast<int64_t>(r) * lds + m;
 #pragma unroll 4
-            for (int s = 0; s < splits; ++s) p += load_scalar<ST>(sp + s * split_stride);   // fixed order
+                for (int s = 0; s < splits; ++s) p += load_scalar<ST>(sp + s * split_stride);   // fixed order
+            }
+            pb[b] = p;
         }
-        // Element pointer of this lane's first chunk; each step moves on by SPW sub-tokens.
-        WT* ptr = out + static_cast<int64_t>(r) * ldo + (static_cast<int64_t>(m0 + sub) * L + q) * 8;
+#pragma unroll
+        for (int b = 0; b < PB; ++b) {
+            const int m0 = (mb0 + b) * 32;
+            if (mb0 + b >= mblocks) break;
+            const float p = pb[b];
+            // Element pointer of this lane's first chunk; each step moves on by SPW sub-tokens.
+            WT* ptr = out + static_cast<int64_t>(r) * ldo + (static_cast<int64_t>(m0 + sub) * L + q) * 8;
 #pragma unroll 8
-        for (int it = 0; it < LPS; ++it, ptr += SPW * L * 8) {
-            const int ms = it * SPW + sub;
-            const float pm = __shfl_sync(kFull, p, ms);
-            if (MODE != 0 && m0 + ms >= M) continue;
+            for (int it = 0; it < LPS; ++it, ptr += SPW * L * 8) {
+                const int ms = it * SPW + sub;
+                const float pm = __shfl_sync(kFull, p, ms);
+                if (MODE != 0 && m0 + ms >= M) continue;
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                float y[8];
+                for (int i = 0; i < CH; ++i) {
+                    float y[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) y[e] = pm * vr[i][e];
-                if (MODE != 2) {
-                    Out8<WT>::store(ptr + i * LPS * 8, y, beta);
-                } else {
-                    const int col = ((m0 + ms) * L + q + LPS * i) * 8;
-                    if (col + 8 <= D) {
+                    for (int e = 0; e < 8; ++e) y[e] = pm * vr[i][e];
+                    if (MODE != 2) {
                         Out8<WT>::store(ptr + i * LPS * 8, y, beta);
                     } else {
+                        const int col = ((m0 + ms) * L + q + LPS * i) * 8;
+                        if (col + 8 <= D) {
+                            Out8<WT>::store(ptr + i * LPS * 8, y, beta);
+                        } else {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            if (col + e < D) {
-                                WT* pe = ptr + i * LPS * 8 + e;
-                                float f = y[e];
-                                if (beta) f += Elem<WT>::load(pe);
-                                Elem<WT>::store(pe, f);
-                            }
+                            for (int e = 0; e < 8; ++e)
+                                if (col + e < D) {
+                                    WT* pe = ptr + i * LPS * 8 + e;
+                                    float f = y[e];
+                                    if (beta) f += Elem<WT>::load(pe);
+                                    Elem<WT>::store(pe, f);
+                                }
+                        }
                     }
                 }
             }
@@ -129,12 +148,24 @@ int launch_mode(int mode, int grid, const void* S, int splits, int64_t split_str
 {
     const ST* s = static_cast<const ST*>(S);
     WT* o = static_cast<WT*>(out);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr = pdl_attribute();
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
     if (mode == 0)
-        expand_rows_vec_kernel<LPS, CH, 0, ST, WT><<<grid, kStreamThreads, 0, stream>>>(s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
+        e = cudaLaunchKernelEx(&cfg, expand_rows_vec_kernel<LPS, CH, 0, ST, WT>, s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
     else if (mode == 1)
-        expand_rows_vec_kernel<LPS, CH, 1, ST, WT><<<grid, kStreamThreads, 0, stream>>>(s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
+        e = cudaLaunchKernelEx(&cfg, expand_rows_vec_kernel<LPS, CH, 1, ST, WT>, s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
     else
-        expand_rows_vec_kernel<LPS, CH, 2, ST, WT><<<grid, kStreamThreads, 0, stream>>>(s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
+        e = cudaLaunchKernelEx(&cfg, expand_rows_vec_kernel<LPS, CH, 2, ST, WT>, s, splits, split_stride, lds, v, R, D, M, mblocks, o, ldo, beta);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return VELORA_ERR_CUDA;
+    }
     return after_launch();
 }
 
@@ -168,7 +199,7 @@ int launch_expand_rows_vec(const void* S, int s_dtype, int splits, int64_t split
     if (L < 1 || L > 128 || (L & (L - 1))) return VELORA_ERR_UNSUPPORTED;
     if (!aligned16(out) || (ldo * static_cast<int64_t>(dtype_size(out_dtype))) % 16) return VELORA_ERR_UNSUPPORTED;
     if (R < 1 || R >= (1 << 30) || lds >= (1 << 30) || D >= (1 << 30)) return VELORA_ERR_UNSUPPORTED;
-    if (s_dtype == VELORA_BF16 && out_dtype != VELORA_BF16) return VELORA_ERR_UNSUPPORTED;
+    if ((s_dtype == VELORA_BF16 || s_dtype == VELORA_FP8_E4M3) && out_dtype != VELORA_BF16) return VELORA_ERR_UNSUPPORTED;
     const int lps = L < 32 ? L : 32, ch = L / lps;
     const int M = static_cast<int>(ceil_div64(D, Dsub));
     const int mblocks = (M + 31) / 32;
@@ -183,6 +214,8 @@ int launch_expand_rows_vec(const void* S, int s_dtype, int splits, int64_t split
     const int r = static_cast<int>(R), d = static_cast<int>(D), ld = static_cast<int>(lds);
     if (s_dtype == VELORA_BF16)
         return launch_shape<__nv_bfloat16, __nv_bfloat16>(lps, ch, mode, grid, S, splits, split_stride, ld, v, r, d, M, mblocks, out, ldo, beta, stream);
+    if (s_dtype == VELORA_FP8_E4M3)
+        return launch_shape<e4m3_t, __nv_bfloat16>(lps, ch, mode, grid, S, splits, split_stride, ld, v, r, d, M, mblocks, out, ldo, beta, stream);
     if (out_dtype == VELORA_BF16)
         return launch_shape<float, __nv_bfloat16>(lps, ch, mode, grid, S, splits, split_stride, ld, v, r, d, M, mblocks, out, ldo, beta, stream);
     return launch_shape<float, float>(lps, ch, mode, grid, S, splits, split_stride, ld, v, r, d, M, mblocks, out, ldo, beta, stream);

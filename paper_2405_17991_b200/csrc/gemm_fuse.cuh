@@ -31,8 +31,8 @@ struct OwnedWalk {
 // `tile` (shared-memory address, 1024-byte aligned).  Adds the row's 64 columns of k-block `kb` into the
 // running inner product `acc` with v (copy in shared memory `sv`, Dsub a power of two >= 8) and stores
 // Z[row, m] whenever a sub-token ends inside the block.  cw = k-blocks per sub-token (1 if Dsub <= 64).
-// Z_BF16 selects the storage type of Z.
-template <bool Z_BF16>
+// ZK selects the storage type of Z: 1 fp32, 2 bf16, 3 E4M3 (the values of the kernels' FUSE parameter).
+template <int ZK>
 __device__ __forceinline__ void compress_kblock(uint32_t tile, int trow, const float* sv, const FuseArgs& fz,
                                                 int cw, int kb, int kblocks, int row, int Mdim, float& acc)
 {
@@ -65,7 +65,8 @@ __device__ __forceinline__ void compress_kblock(uint32_t tile, int trow, const f
         if (jv + 8 == Dsub || (kb == kblocks - 1 && c == 7)) {
             const int m = (kb * BK + c * 8) / Dsub;
             if (row < Mdim && m < fz.M) {
-                if (Z_BF16) static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
+                if (ZK == 2) static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(acc);
+                else if (ZK == 3) static_cast<e4m3_t*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = float_to_e4m3(acc);
                 else static_cast<float*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = acc;
             }
         }

@@ -108,6 +108,11 @@ int launch_gemm_simt(const void* A, int a_dtype, int64_t a_sm, int64_t a_sk,
     const int64_t gx = ceil_div64(Ndim, TN), gy = ceil_div64(Mdim, TM);
     if (gy > 65535) return VELORA_ERR_UNSUPPORTED;
     dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(gy));
+    if (b_dtype == VELORA_FP8_E4M3) {                    // Z in its 8-bit store as the second operand of dY^T Z
+        if (a_dtype == VELORA_BF16)
+            return dispatch_c<__nv_bfloat16, e4m3_t>(A, a_sm, a_sk, B, b_sn, b_sk, C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, grid, stream);
+        return dispatch_c<float, e4m3_t>(A, a_sm, a_sk, B, b_sn, b_sk, C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, grid, stream);
+    }
     if (a_dtype == VELORA_BF16 && b_dtype == VELORA_BF16)
         return dispatch_c<__nv_bfloat16, __nv_bfloat16>(A, a_sm, a_sk, B, b_sn, b_sk, C, c_dtype, ldc, beta, Mdim, Ndim, Kdim, grid, stream);
     if (a_dtype == VELORA_BF16 && b_dtype == VELORA_F32)

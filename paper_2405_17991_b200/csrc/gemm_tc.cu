@@ -211,7 +211,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!own.owned()) continue;
                 if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
                 ++oc;
-                compress_kblock<FUSE == 2>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
+                compress_kblock<FUSE>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
                 __syncwarp();                                 // every lane's reads of the tile are done
                 if (lane == 0) mbar_arrive(cempty);
             }
@@ -280,15 +280,15 @@ template <bool A_MN, bool B_MN, typename CT, int FUSE = 0>
 int launch_kernel(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t ldc, int beta,
                   int Mdim, int Ndim, int Kdim, int* status, cudaStream_t stream, const FuseArgs fz = FuseArgs{})
 {
-    static bool configured[64] = {};
+    static DeviceOnce configured;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
     auto kern = gemm_tc_kernel<A_MN, B_MN, CT, FUSE>;
-    if (!configured[dev]) {
+    if (!configured.get(dev)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(FUSE ? FUSE_SMEM : GEMM_SMEM)) != cudaSuccess)
             return VELORA_ERR_CUDA;
-        configured[dev] = true;
+        configured.set(dev);
     }
     DeviceInfo di;
     int rc = device_info(&di);
@@ -414,6 +414,8 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
         const int m = static_cast<int>(N), n = static_cast<int>(O), k = static_cast<int>(D);
         if (z_dtype == VELORA_F32)
             return launch_kernel<false, false, __nv_bfloat16, 1>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);
+        if (z_dtype == VELORA_FP8_E4M3)
+            return launch_kernel<false, false, __nv_bfloat16, 3>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);
         return launch_kernel<false, false, __nv_bfloat16, 2>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);
     }
     int rc = launch_gemm_tc(GEMM_NT_K_K, X, ldx, W, ldw, Y, dtype, ldy, 0, N, O, D, dtype, status, stream);

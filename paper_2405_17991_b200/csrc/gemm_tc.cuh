@@ -54,13 +54,16 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
                              void* Y, int64_t ldy, void* Z, int z_dtype, int64_t ldz,
                              int dtype, int64_t N, int64_t D, int64_t O, int Dsub, int* status, cudaStream_t stream);
 
-// TMA-staged streaming kernels (stream_tma.cu): X tiles flow through a shared-memory ring.
+// Row-streaming kernels (stream_rows.cu): bf16 X with 16-byte aligned rows, Dsub = 8 * 2^k up to 1024.
 // Return VELORA_ERR_UNSUPPORTED (nothing launched) when the shape does not fit them.
-int launch_compress_tma(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
-                        void* Z, int z_dtype, int64_t ldz, int* status, cudaStream_t stream);
-int launch_init_v_partials_tma(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub,
-                               float* partials, int max_partials, int* num_partials, int* status,
-                               cudaStream_t stream);
+int launch_compress_rows(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                         void* Z, int z_dtype, int64_t ldz, cudaStream_t stream);
+int launch_init_v_partials_rows(const void* X, int64_t N, int64_t D, int64_t ldx, int Dsub,
+                                float* partials, int max_partials, int* num_partials, cudaStream_t stream);
+
+// One tiny CTA whose bounded waits run out (limit_ns for the first, the abort flag for the second); raises
+// `status` (may be NULL) and the per-device error word like a real kernel would.  observed[4]: device ints.
+int launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, int* observed, cudaStream_t stream);
 
 // Reads (synchronising `stream`) and clears the device word in which the streaming kernels record an
 // expired wait: VELORA_OK or VELORA_ERR_TIMEOUT.

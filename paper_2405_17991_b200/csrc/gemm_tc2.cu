@@ -278,7 +278,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!own.owned()) continue;
                 if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
                 ++oc;
-                compress_kblock<FUSE == 2>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
+                compress_kblock<FUSE>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
                 __syncwarp();                                // every lane's reads of the tile are done
                 if (lane == 0) mbar_arrive(cempty);
             }
@@ -331,14 +331,14 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, void* C, int64_t l
                 const FuseArgs fz = FuseArgs{})
 {
     constexpr size_t smem_bytes = FUSE ? P_FUSE_SMEM : P_SMEM;
-    static bool configured[64] = {};
+    static DeviceOnce configured;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
     auto kern = gemm_pair_kernel<A_MN, B_MN, CT, FUSE>;
-    if (!configured[dev]) {
+    if (!configured.get(dev)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) != cudaSuccess)
             return VELORA_ERR_CUDA;
-        configured[dev] = true;
+        configured.set(dev);
     }
     const int tiles_m = (Mdim + 2 * P_BM - 1) / (2 * P_BM), tiles_n = (Ndim + P_BN - 1) / P_BN;
     const int64_t tiles = static_cast<int64_t>(tiles_m) * tiles_n;
@@ -419,6 +419,8 @@ int launch_linear_forward_tc_pair(const void* X, int64_t ldx, const void* W, int
     const int m = static_cast<int>(N), n = static_cast<int>(O), k = static_cast<int>(D);
     if (z_dtype == VELORA_F32)
         return launch_pair<false, false, __nv_bfloat16, 1>(ta, tb, Y, ldy, 0, m, n, k, status, di.sm_count, stream, fz);
+    if (z_dtype == VELORA_FP8_E4M3)
+        return launch_pair<false, false, __nv_bfloat16, 3>(ta, tb, Y, ldy, 0, m, n, k, status, di.sm_count, stream, fz);
     return launch_pair<false, false, __nv_bfloat16, 2>(ta, tb, Y, ldy, 0, m, n, k, status, di.sm_count, stream, fz);
 }
 

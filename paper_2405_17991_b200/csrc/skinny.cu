@@ -450,7 +450,10 @@ int launch_weight_grad_skinny(const void* dY, int dy_dtype, int64_t N, int64_t O
     float* P = reinterpret_cast<float*>(static_cast<char*>(ws) + p.partial_bytes);
     const int n = static_cast<int>(N), o = static_cast<int>(O);
     int rc;
-    if (dy_dtype == VELORA_BF16)
+    if (z_dtype == VELORA_FP8_E4M3)
+        rc = dy_dtype == VELORA_BF16 ? launch_partial<__nv_bfloat16, e4m3_t>(p, dY, lddy, Z, ldz, n, o, partials, stream)
+                                     : launch_partial<float, e4m3_t>(p, dY, lddy, Z, ldz, n, o, partials, stream);
+    else if (dy_dtype == VELORA_BF16)
         rc = z_dtype == VELORA_BF16 ? launch_partial<__nv_bfloat16, __nv_bfloat16>(p, dY, lddy, Z, ldz, n, o, partials, stream)
                                     : launch_partial<__nv_bfloat16, float>(p, dY, lddy, Z, ldz, n, o, partials, stream);
     else
@@ -477,6 +480,7 @@ int launch_linear_forward_skinny(const void* X, int64_t ldx, const void* W, int6
 {
     const bool pow2 = Dsub >= 8 && Dsub <= VELORA_MAX_DSUB && (Dsub & (Dsub - 1)) == 0;
     if (!pow2 || O < 1 || O > 64 || N < 1 || N > (1 << 30) || D > (1 << 30)) return VELORA_ERR_UNSUPPORTED;
+    if (z_dtype == VELORA_FP8_E4M3) return VELORA_ERR_UNSUPPORTED;     // 8-bit Z: product, then the compress kernel
     if (!tc_operand_ok(X, ldx) || !tc_operand_ok(W, ldw)) return VELORA_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = device_info(&di);
@@ -494,14 +498,14 @@ int launch_linear_forward_skinny(const void* X, int64_t ldx, const void* W, int6
     // One box for four 64-column tiles needs whole 64-column chunks; otherwise four two-dimensional boxes.
     int use3d = (D % SF_BK == 0 && make_tmap_bf16_chunks3d(&tx3, X, D, N, ldx, SF_TOKENS, SF_SB) == VELORA_OK) ? 1 : 0;
     if (!use3d) tx3 = tx;
-    static bool configured[64] = {};
+    static DeviceOnce configured;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
-    if (!configured[dev]) {
+    if (!configured.get(dev)) {
         if (cudaFuncSetAttribute(skinny_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SF_SMEM)) != cudaSuccess ||
             cudaFuncSetAttribute(skinny_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SF_SMEM)) != cudaSuccess)
             return VELORA_ERR_CUDA;
-        configured[dev] = true;
+        configured.set(dev);
     }
     FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>(ceil_div64(D, Dsub))};
     const int grid = static_cast<int>(ceil_div64(N, SF_TOKENS));

@@ -1,17 +1,9 @@
 // HBM-bound streaming kernels of the VeLoRA path: init_v, compress, reconstruct and the expansion
 // of the factored weight gradient (arxiv 2405.17991, Section 3.1 Eq. 1 / Eq. 2, Section 3.2).
 //
-// Vector kernels.  A row of X is a sequence of 16-byte chunks (8 bf16).  A sub-token of length
-// Dsub = 8*L is covered by LPS = min(L, 32) adjacent lanes, each lane owning CH = L / LPS chunks, so
-// a warp instruction touches one contiguous 512-byte span.  Work items (row, m, lane-in-group) are
-// numbered row-major and walked with a grid-wide stride that is a multiple of 32: a thread keeps the
-// same position inside its sub-token for the whole kernel and holds its slice of v in registers.  The
-// walk carries (row, pos) incrementally in 32-bit integers -- no division, no 64-bit multiply in the
-// loop (the host cuts very large inputs into launches whose offsets fit 31 bits).  Loads are software
-// pipelined: the next batch of 16-byte loads is issued before the current batch is reduced, so a
-// thread always has loads in flight.  When Dsub does not divide D the last sub-token's missing chunks
-// are not loaded (zero extension); that case uses the RAGGED instances, the common case carries no
-// bounds checks on columns.
+// The common case (bf16 rows that are 16-byte aligned, Dsub = 8 * 2^k) is served by stream_rows.cu
+// (compress, init_v) and expand_kernels.cu (reconstruct, expansion of the factored weight gradient).  This
+// file holds the kernels for everything else and the routing between all of them.
 //
 // Element kernels cover everything else (fp32 data, Dsub not a multiple of 8, unaligned rows) with
 // the same arithmetic, one element per lane.
@@ -24,67 +16,10 @@ namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
 
-// Walks items tid, tid + S, tid + 2S, ... as (row, pos), pos in [0, items_per_row).
-struct ItemWalk {
-    int row, pos;
-    int row_step, pos_step, ipr;
-    __device__ __forceinline__ void init(int items_per_row)
-    {
-        const int tid = blockIdx.x * blockDim.x + threadIdx.x;
-        const int S = gridDim.x * blockDim.x;
-        ipr = items_per_row;
-        row = tid / ipr;
-        pos = tid - row * ipr;
-        row_step = S / ipr;
-        pos_step = S - row_step * ipr;
-    }
-    __device__ __forceinline__ void advance()
-    {
-        pos += pos_step;
-        row += row_step;
-        if (pos >= ipr) { pos -= ipr; ++row; }
-    }
-};
-
-__device__ __forceinline__ void unpack8(const uint4& c, float (&x)[8])
-{
-    x[0] = bf16_lo(c.x); x[1] = bf16_hi(c.x);
-    x[2] = bf16_lo(c.y); x[3] = bf16_hi(c.y);
-    x[4] = bf16_lo(c.z); x[5] = bf16_hi(c.z);
-    x[6] = bf16_lo(c.w); x[7] = bf16_hi(c.w);
-}
-
-// Loads chunk `chunk` of a row, zeroing whatever lies at or beyond column D.
-__device__ __forceinline__ uint4 load_chunk_ragged(const uint4* row_ptr, int chunk, int D)
-{
-    const int col = chunk * 8;
-    uint4 c = make_uint4(0u, 0u, 0u, 0u);
-    if (col < D) {
-        c = __ldg(row_ptr + chunk);
-        if (col + 8 > D) {                       // ragged end of a row whose width is not a multiple of 8
-            const int keep = D - col;            // 1..7 valid elements
-            uint32_t w[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (2 * i >= keep) w[i] = 0u;
-                else if (2 * i + 1 >= keep) w[i] &= 0x0000ffffu;
-            }
-            c = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-    }
-    return c;
-}
-
-template <bool RAGGED>
-__device__ __forceinline__ uint4 load_chunk(const uint4* row_ptr, int chunk, int D)
-{
-    if (RAGGED) return load_chunk_ragged(row_ptr, chunk, D);
-    return __ldg(row_ptr + chunk);
-}
-
 template <typename ZT> __device__ __forceinline__ void store_z(ZT* p, float z);
 template <> __device__ __forceinline__ void store_z<float>(float* p, float z) { *p = z; }
 template <> __device__ __forceinline__ void store_z<__nv_bfloat16>(__nv_bfloat16* p, float z) { *p = __float2bfloat16_rn(z); }
+template <> __device__ __forceinline__ void store_z<e4m3_t>(e4m3_t* p, float z) { *p = float_to_e4m3(z); }
 
 template <typename ZT> __device__ __forceinline__ float load_z(const ZT* p);
 template <> __device__ __forceinline__ float load_z<float>(const float* p) { return __ldg(p); }
@@ -92,130 +27,7 @@ template <> __device__ __forceinline__ float load_z<__nv_bfloat16>(const __nv_bf
 {
     return __bfloat162float(*p);
 }
-
-// ------------------------------------------------------------------ compress (vector)
-template <int LPS, int CH, int U, bool RAGGED, typename ZT>
-__global__ void __launch_bounds__(kStreamThreads)
-compress_vec_kernel(const uint4* __restrict__ X, int N, int D, int ldx_chunks, int M,
-                    const float* __restrict__ v, ZT* __restrict__ Z, int ldz)
-{
-    constexpr int L = LPS * CH;                  // chunks per sub-token
-    const int q = threadIdx.x & (LPS - 1);       // fixed position inside the sub-token
-    float vr[CH][8];
-#pragma unroll
-    for (int i = 0; i < CH; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) vr[i][e] = __ldg(v + 8 * (q + LPS * i) + e);
-
-    ItemWalk w;
-    w.init(M * LPS);
-    // One batch = U items per thread; zoff is the item's offset in Z, or -1 past the end.
-    auto fetch = [&](uint4 (&d)[U][CH], int (&zoff)[U]) {
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const bool valid = w.row < N;
-            const int m = w.pos / LPS;           // LPS is a power of two
-            zoff[u] = valid ? w.row * ldz + m : -1;
-            const uint4* rp = X + (valid ? w.row * ldx_chunks : 0);
-#pragma unroll
-            for (int i = 0; i < CH; ++i)
-                d[u][i] = valid ? load_chunk<RAGGED>(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
-            w.advance();
-        }
-    };
-    uint4 cur[U][CH];
-    int czoff[U];
-    fetch(cur, czoff);
-    while (__any_sync(kFull, czoff[0] >= 0)) {
-        uint4 nxt[U][CH];
-        int nzoff[U];
-        fetch(nxt, nzoff);                       // next batch in flight while this one is reduced
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float acc = 0.f;
-#pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                float x[8];
-                unpack8(cur[u][i], x);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc = fmaf(x[e], vr[i][e], acc);
-            }
-#pragma unroll
-            for (int off = LPS / 2; off >= 1; off >>= 1) acc += __shfl_xor_sync(kFull, acc, off);
-            if (q == 0 && czoff[u] >= 0) store_z<ZT>(Z + czoff[u], acc);
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            czoff[u] = nzoff[u];
-#pragma unroll
-            for (int i = 0; i < CH; ++i) cur[u][i] = nxt[u][i];
-        }
-    }
-}
-
-// ------------------------------------------------------------------ init_v (vector): per-CTA partial sums
-template <int LPS, int CH, int U, bool RAGGED>
-__global__ void __launch_bounds__(kStreamThreads)
-init_v_partial_vec_kernel(const uint4* __restrict__ X, int N, int D, int ldx_chunks, int M,
-                          float* __restrict__ partials /* [gridDim.x][8*L] */)
-{
-    constexpr int L = LPS * CH;
-    constexpr int W = 8 * CH;                    // accumulators per thread
-    const int q = threadIdx.x & (LPS - 1);
-    float acc[CH][8];
-#pragma unroll
-    for (int i = 0; i < CH; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[i][e] = 0.f;
-
-    ItemWalk w;
-    w.init(M * LPS);
-    auto fetch = [&](uint4 (&d)[U][CH]) -> bool {
-        const bool any = w.row < N;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const bool valid = w.row < N;
-            const uint4* rp = X + (valid ? w.row * ldx_chunks : 0);
-            const int m = w.pos / LPS;
-#pragma unroll
-            for (int i = 0; i < CH; ++i)
-                d[u][i] = valid ? load_chunk<RAGGED>(rp, m * L + q + LPS * i, D) : make_uint4(0u, 0u, 0u, 0u);
-            w.advance();
-        }
-        return any;
-    };
-    uint4 cur[U][CH];
-    bool more = fetch(cur);
-    while (more) {
-        uint4 nxt[U][CH];
-        more = fetch(nxt);
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-#pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                float x[8];
-                unpack8(cur[u][i], x);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[i][e] += x[e];
-                cur[u][i] = nxt[u][i];
-            }
-    }
-
-    // Fixed-order reduction over the threads of the CTA that share a position q.
-    extern __shared__ float sacc[];              // [kStreamThreads][W]
-#pragma unroll
-    for (int i = 0; i < CH; ++i)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) sacc[threadIdx.x * W + i * 8 + e] = acc[i][e];
-    __syncthreads();
-    for (int j = threadIdx.x; j < 8 * L; j += kStreamThreads) {
-        const int chunk = j >> 3, e = j & 7;
-        const int qq = chunk % LPS, i = chunk / LPS;
-        float s = 0.f;
-        for (int t = qq; t < kStreamThreads; t += LPS) s += sacc[t * W + i * 8 + e];
-        partials[static_cast<int64_t>(blockIdx.x) * (8 * L) + j] = s;
-    }
-}
+template <> __device__ __forceinline__ float load_z<e4m3_t>(const e4m3_t* p) { return e4m3_to_float(*p); }
 
 // ------------------------------------------------------------------ init_v (element-wise) partial sums
 // CTA b owns rows [b*rows_per_cta, ...).  For each block of up to 256 positions j, thread t adds
@@ -631,25 +443,6 @@ expand_any_kernel(const ST* __restrict__ S, int splits, int64_t split_stride, in
 }
 
 // ------------------------------------------------------------------ host side
-struct VecShape {
-    bool ok;
-    int lps, ch, u;
-};
-
-// Vector kernels need Dsub = 8 * L with L a power of two up to 128.
-VecShape vec_shape(int Dsub)
-{
-    VecShape s{false, 0, 0, 0};
-    if (Dsub % 8) return s;
-    const int L = Dsub / 8;
-    if (L < 1 || L > 128 || (L & (L - 1))) return s;
-    s.ok = true;
-    s.lps = L < 32 ? L : 32;
-    s.ch = L / s.lps;
-    s.u = s.ch == 1 ? 4 : (s.ch == 2 ? 2 : 1);
-    return s;
-}
-
 bool rows_vectorisable(const void* p, int64_t ld_elems)
 {
     return aligned16(p) && (ld_elems % 8 == 0);
@@ -672,30 +465,6 @@ int check_launch()
 {
     return after_launch();
 }
-
-// Largest number of rows one vector launch may take so that item counts and the element offsets
-// row*ld_a, row*ld_b stay within 31 bits.
-int64_t max_rows_per_launch(int items_per_row, int64_t ld_a, int64_t ld_b)
-{
-    int64_t r = (static_cast<int64_t>(1) << 30) / items_per_row;
-    const int64_t lim = (static_cast<int64_t>(1) << 31) - 1;
-    if (ld_a > 0 && lim / ld_a < r) r = lim / ld_a;
-    if (ld_b > 0 && lim / ld_b < r) r = lim / ld_b;
-    return r < 1 ? 1 : r;
-}
-
-#define VELORA_DISPATCH_VEC(SHAPE, KERNEL_CALL)                                              \
-    switch ((SHAPE).lps * 8 + (SHAPE).ch) {                                                  \
-        case 1 * 8 + 1: { KERNEL_CALL(1, 1, 4); break; }                                     \
-        case 2 * 8 + 1: { KERNEL_CALL(2, 1, 4); break; }                                     \
-        case 4 * 8 + 1: { KERNEL_CALL(4, 1, 4); break; }                                     \
-        case 8 * 8 + 1: { KERNEL_CALL(8, 1, 4); break; }                                     \
-        case 16 * 8 + 1: { KERNEL_CALL(16, 1, 4); break; }                                   \
-        case 32 * 8 + 1: { KERNEL_CALL(32, 1, 4); break; }                                   \
-        case 32 * 8 + 2: { KERNEL_CALL(32, 2, 2); break; }                                   \
-        case 32 * 8 + 4: { KERNEL_CALL(32, 4, 1); break; }                                   \
-        default: return VELORA_ERR_UNSUPPORTED;                                              \
-    }
 
 }  // namespace
 
@@ -749,34 +518,13 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
     int* status = static_cast<int*>(ws) + 1;             // word 1: degenerate-sum flag of this call
     float* partials = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
     const int M = static_cast<int>(ceil_div64(D, Dsub));
-    const VecShape vs = vec_shape(Dsub);
-    const bool ragged = (D % Dsub) != 0;
     int num_partials = 0;
 
-    int tma_rc = VELORA_ERR_UNSUPPORTED;
-    if (x_dtype == VELORA_BF16 && D >= 256)
-        tma_rc = launch_init_v_partials_tma(X, N, D, ldx, Dsub, partials, kInitVMaxCtas, &num_partials, nullptr, stream);
-    if (tma_rc != VELORA_ERR_UNSUPPORTED) {
-        if (tma_rc != VELORA_OK) return tma_rc;
-    } else if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx) &&
-        N <= max_rows_per_launch(M * vs.lps, ldx / 8, 0)) {
-        const int64_t items = N * M * vs.lps;
-        int grid = 0;
-        int rc = stream_grid(items, 2 * vs.u, &grid);
-        if (rc != VELORA_OK) return rc;
-        if (grid > kInitVMaxCtas) grid = kInitVMaxCtas;
-        num_partials = grid;
-        const size_t smem = static_cast<size_t>(kStreamThreads) * 8 * vs.ch * sizeof(float);
-        const int n = static_cast<int>(N), d = static_cast<int>(D), ldc = static_cast<int>(ldx / 8);
-#define CALL_INIT(LPS, CH, U)                                                                             \
-        if (ragged)                                                                                       \
-            init_v_partial_vec_kernel<LPS, CH, U, true><<<grid, kStreamThreads, smem, stream>>>(          \
-                static_cast<const uint4*>(X), n, d, ldc, M, partials);                                    \
-        else                                                                                              \
-            init_v_partial_vec_kernel<LPS, CH, U, false><<<grid, kStreamThreads, smem, stream>>>(         \
-                static_cast<const uint4*>(X), n, d, ldc, M, partials)
-        VELORA_DISPATCH_VEC(vs, CALL_INIT)
-#undef CALL_INIT
+    int rows_rc = VELORA_ERR_UNSUPPORTED;
+    if (x_dtype == VELORA_BF16)
+        rows_rc = launch_init_v_partials_rows(X, N, D, ldx, Dsub, partials, kInitVMaxCtas, &num_partials, stream);
+    if (rows_rc != VELORA_ERR_UNSUPPORTED) {
+        if (rows_rc != VELORA_OK) return rows_rc;
     } else {
         DeviceInfo di;
         int rc = device_info(&di);
@@ -805,13 +553,12 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
                     const float* v, void* Z, int z_dtype, int64_t ldz, cudaStream_t stream)
 {
     const int M = static_cast<int>(ceil_div64(D, Dsub));
-    const VecShape vs = vec_shape(Dsub);
-    const bool ragged = (D % Dsub) != 0;
-    if (x_dtype == VELORA_BF16 && D >= 256) {            // TMA-staged kernel: large rows, Dsub in {8..256}
-        const int rc = launch_compress_tma(X, N, D, ldx, Dsub, v, Z, z_dtype, ldz, nullptr, stream);
+    if (x_dtype == VELORA_BF16) {                        // aligned rows, Dsub = 8 * 2^k: the row-streaming kernel
+        const int rc = launch_compress_rows(X, N, D, ldx, Dsub, v, Z, z_dtype, ldz, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     }
-    if (x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && rows_vectorisable(X, ldx) && D < (1 << 30)) {
+    const bool z8 = z_dtype == VELORA_FP8_E4M3;          // 8-bit Z: the TMA kernel above or the element kernel below
+    if (!z8 && x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && rows_vectorisable(X, ldx) && D < (1 << 30)) {
         int grid = 0;
         const int rc = stream_grid(N * ceil_div64(D, 8), 4, &grid);
         if (rc != VELORA_OK) return rc;
@@ -826,34 +573,7 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
 #undef CALL_SMALL
         return check_launch();
     }
-    if (x_dtype == VELORA_BF16 && vs.ok && rows_vectorisable(X, ldx)) {
-        const int64_t step = max_rows_per_launch(M * vs.lps, ldx / 8, ldz);
-        const int d = static_cast<int>(D), ldc = static_cast<int>(ldx / 8), ldzi = static_cast<int>(ldz);
-        for (int64_t r0 = 0; r0 < N; r0 += step) {
-            const int n = static_cast<int>((N - r0 < step) ? N - r0 : step);
-            int grid = 0;
-            int rc = stream_grid(static_cast<int64_t>(n) * M * vs.lps, 2 * vs.u, &grid);
-            if (rc != VELORA_OK) return rc;
-            const uint4* xp = static_cast<const uint4*>(X) + r0 * (ldx / 8);
-#define CALL_COMPRESS_T(LPS, CH, U, RAG, ZT)                                                              \
-            compress_vec_kernel<LPS, CH, U, RAG, ZT><<<grid, kStreamThreads, 0, stream>>>(                \
-                xp, n, d, ldc, M, v, static_cast<ZT*>(Z) + r0 * ldz, ldzi)
-#define CALL_COMPRESS(LPS, CH, U)                                                                         \
-            if (z_dtype == VELORA_F32) {                                                                  \
-                if (ragged) CALL_COMPRESS_T(LPS, CH, U, true, float);                                     \
-                else CALL_COMPRESS_T(LPS, CH, U, false, float);                                           \
-            } else {                                                                                      \
-                if (ragged) CALL_COMPRESS_T(LPS, CH, U, true, __nv_bfloat16);                             \
-                else CALL_COMPRESS_T(LPS, CH, U, false, __nv_bfloat16);                                   \
-            }
-            VELORA_DISPATCH_VEC(vs, CALL_COMPRESS)
-#undef CALL_COMPRESS
-#undef CALL_COMPRESS_T
-            if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
-        }
-        return VELORA_OK;
-    }
-    if (x_dtype == VELORA_BF16 && Dsub % 8 == 0 && rows_vectorisable(X, ldx) && N < (1 << 30) && D < (1 << 28)) {
+    if (!z8 && x_dtype == VELORA_BF16 && Dsub % 8 == 0 && rows_vectorisable(X, ldx) && N < (1 << 30) && D < (1 << 28)) {
         // any other multiple of 8 (96, 48, 24 ...): segmented reduction over the lanes of a sub-token
         int sgrid = 0;
         const int src = stream_grid(N * 32, 1, &sgrid);
@@ -875,8 +595,10 @@ int launch_compress(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ld
     compress_elem_kernel<XT, ZT><<<grid, kStreamThreads, 0, stream>>>(                                    \
         static_cast<const XT*>(X), N, static_cast<int>(D), ldx, Dsub, M, v, static_cast<ZT*>(Z), ldz)
     if (x_dtype == VELORA_BF16 && z_dtype == VELORA_F32) CALL_ELEM(__nv_bfloat16, float);
+    else if (x_dtype == VELORA_BF16 && z8) CALL_ELEM(__nv_bfloat16, e4m3_t);
     else if (x_dtype == VELORA_BF16) CALL_ELEM(__nv_bfloat16, __nv_bfloat16);
     else if (z_dtype == VELORA_F32) CALL_ELEM(float, float);
+    else if (z8) CALL_ELEM(float, e4m3_t);
     else CALL_ELEM(float, __nv_bfloat16);
 #undef CALL_ELEM
     return check_launch();
@@ -914,7 +636,8 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
         const int rc = launch_expand_rows_vec(Z, z_dtype, 1, 0, ldz, v, N, D, Dsub, Xhat, x_dtype, ldxhat, 0, stream);
         if (rc != VELORA_ERR_UNSUPPORTED) return rc;
     }
-    if (x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && D % 8 == 0 && rows_vectorisable(Xhat, ldxhat) &&
+    const bool z8 = z_dtype == VELORA_FP8_E4M3;          // 8-bit Z: the vector expansion above or the element kernel below
+    if (!z8 && x_dtype == VELORA_BF16 && (Dsub == 1 || Dsub == 2 || Dsub == 4) && D % 8 == 0 && rows_vectorisable(Xhat, ldxhat) &&
         D < (1 << 30)) {
         const int M = static_cast<int>(ceil_div64(D, Dsub));
         int grid = 0;
@@ -931,7 +654,7 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
 #undef CALL_SMALL
         return check_launch();
     }
-    {
+    if (!z8) {
         const int arc = launch_expand_any(Z, z_dtype, 1, 0, ldz, v, N, D, Dsub, Xhat, x_dtype, ldxhat, 0, stream);
         if (arc != VELORA_ERR_UNSUPPORTED) return arc;
     }
@@ -943,6 +666,8 @@ int launch_reconstruct(const void* Z, int z_dtype, int64_t ldz, int64_t N, int64
         static_cast<const ZT*>(Z), ldz, N, static_cast<int>(D), Dsub, v, static_cast<XT*>(Xhat), ldxhat)
     if (z_dtype == VELORA_F32 && x_dtype == VELORA_BF16) CALL_ELEM(float, __nv_bfloat16);
     else if (z_dtype == VELORA_F32) CALL_ELEM(float, float);
+    else if (z8 && x_dtype == VELORA_BF16) CALL_ELEM(e4m3_t, __nv_bfloat16);
+    else if (z8) CALL_ELEM(e4m3_t, float);
     else if (x_dtype == VELORA_BF16) CALL_ELEM(__nv_bfloat16, __nv_bfloat16);
     else CALL_ELEM(__nv_bfloat16, float);
 #undef CALL_ELEM
@@ -970,6 +695,74 @@ int launch_expand_p(const float* P, int splits, int64_t split_stride, int64_t ld
 }
 
 }  // namespace velora
+// ------------------------------------------------------------------ scale of the 8-bit Z store
+namespace velora {
+namespace {
+
+// Largest |z| of a contiguous fp32 array, as the bit pattern of a non-negative float (those order like
+// unsigned integers; a NaN's pattern is above every finite one, so it surfaces as "not finite").
+__global__ void __launch_bounds__(kStreamThreads) z_amax_kernel(const float* __restrict__ Z, int64_t count, unsigned int* amax_bits)
+{
+    unsigned int best = 0u;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kStreamThreads;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kStreamThreads + threadIdx.x; i < count; i += stride) {
+        const unsigned int b = __float_as_uint(__ldg(Z + i)) & 0x7fffffffu;
+        best = b > best ? b : best;
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned int o = __shfl_xor_sync(kFull, best, off);
+        best = o > best ? o : best;
+    }
+    if ((threadIdx.x & 31) == 0 && best) atomicMax(amax_bits, best);     // a maximum: the order of arrival does not matter
+}
+
+__global__ void __launch_bounds__(kStreamThreads) z8_scale_kernel(const unsigned int* amax_bits, float headroom, const float* __restrict__ v,
+                                                                   int Dsub, float* zscale, float* v_store, float* v_load)
+{
+    const float amax = __uint_as_float(*amax_bits);
+    float scale = 1.f;
+    if (amax > 0.f && amax <= 3.0e38f) scale = headroom * amax / 448.f;
+    if (!(scale > 0.f) || !(scale <= 3.0e38f)) scale = 1.f;
+    if (threadIdx.x == 0) *zscale = scale;
+    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) {
+        const float x = __ldg(v + j);
+        v_store[j] = x / scale;
+        v_load[j] = x * scale;
+    }
+}
+
+}  // namespace
+
+size_t z8_calibrate_workspace_bytes(int64_t N, int64_t D, int Dsub)
+{
+    const size_t zbytes = static_cast<size_t>(N) * static_cast<size_t>(ceil_div64(D, Dsub)) * sizeof(float);
+    return kStatusBytes + 256 + (zbytes + 255) / 256 * 256;
+}
+
+int launch_z8_calibrate(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx, int Dsub, const float* v,
+                        float headroom, float* zscale, float* v_store, float* v_load,
+                        void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (ws_bytes < z8_calibrate_workspace_bytes(N, D, Dsub)) return VELORA_ERR_WORKSPACE;
+    unsigned int* amax_bits = reinterpret_cast<unsigned int*>(static_cast<char*>(ws) + kStatusBytes);
+    float* Z = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes + 256);
+    const int64_t M = ceil_div64(D, Dsub);
+    if (cudaMemsetAsync(amax_bits, 0, sizeof(unsigned int), stream) != cudaSuccess) return VELORA_ERR_CUDA;
+    if (N > 0) {
+        int rc = launch_compress(X, x_dtype, N, D, ldx, Dsub, v, Z, VELORA_F32, M, stream);
+        if (rc != VELORA_OK) return rc;
+        int grid = 0;
+        rc = stream_grid(N * M, 4, &grid);
+        if (rc != VELORA_OK) return rc;
+        z_amax_kernel<<<grid, kStreamThreads, 0, stream>>>(Z, N * M, amax_bits);
+        if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
+    }
+    z8_scale_kernel<<<1, kStreamThreads, 0, stream>>>(amax_bits, headroom, v, Dsub, zscale, v_store, v_load);
+    return check_launch();
+}
+
+}  // namespace velora
 // ------------------------------------------------------------------ velora_init_v without a workspace
 // Scratch for velora_init_v_static: the status header plus one row of partial sums per CTA, for
 // sub-tokens of up to VELORA_INIT_V_STATIC_MAX_DSUB elements.  It is part of the loaded module, so
@@ -985,16 +778,16 @@ static __device__ __align__(256) unsigned char g_init_v_scratch[kStaticScratchBy
 // device, with that device current, and remembered.
 int static_scratch_address(void** out)
 {
-    static void* cached[64] = {};
+    static std::atomic<void*> cached[64];          // two threads' first calls both store the same address
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return VELORA_ERR_CUDA;
     if (dev < 0 || dev >= 64) return VELORA_ERR_UNSUPPORTED;
-    if (!cached[dev]) {
-        void* p = nullptr;
+    void* p = cached[dev].load(std::memory_order_relaxed);
+    if (!p) {
         if (cudaGetSymbolAddress(&p, g_init_v_scratch) != cudaSuccess || !p) return VELORA_ERR_CUDA;
-        cached[dev] = p;
+        cached[dev].store(p, std::memory_order_relaxed);
     }
-    *out = cached[dev];
+    *out = p;
     return VELORA_OK;
 }
 }  // namespace

@@ -55,10 +55,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Waits for the phase with the given parity to complete.  Never spins for ever: returns false when
-// another role has raised `abort_flag` or after kWaitLimitNs; the caller then raises the flag itself,
-// records the failure and leaves its loop.
+// another role has raised `abort_flag` or after `limit_ns` (kWaitLimitNs everywhere but in the self-test of
+// this very path); the caller then raises the flag itself, records the failure and leaves its loop.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t backoff_ns = 0)
+                                          uint32_t backoff_ns = 0, unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         // probe made a sleeping waiter notice its barrier about a microsecond late.
         if ((++spins & (backoff_ns ? 15u : 63u)) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+            if (globaltimer_ns() - t0 > limit_ns) return false;
         }
     }
     return true;
@@ -81,10 +81,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // with a single probe each, which also gives every lane its own acquire of the data the phase covers.
 // Keeps 31 of 32 lanes from polling shared memory while the tensor cores stream operands out of it.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                               uint32_t backoff_ns = 0)
+                                               uint32_t backoff_ns = 0, unsigned long long limit_ns = kWaitLimitNs)
 {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, backoff_ns) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, backoff_ns, limit_ns) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (ok) {
         for (int i = 0; i < 1024 && !mbar_try_wait(bar, parity); ++i) {}

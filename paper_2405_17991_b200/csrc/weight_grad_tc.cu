@@ -424,14 +424,14 @@ template <bool CLUSTER, int LPS, int CH, typename WT>
 int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, const WgPlan& p, int smem_optin,
               cudaStream_t stream)
 {
-    static bool configured[64] = {};
+    static DeviceOnce configured;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
     auto kern = wg_kernel<CLUSTER, LPS, CH, WT>;
-    if (!configured[dev]) {
+    if (!configured.get(dev)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
             return VELORA_ERR_CUDA;
-        configured[dev] = true;
+        configured.set(dev);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(p.tiles_o), static_cast<unsigned>(p.splits), 1);
@@ -496,6 +496,9 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
         if (z_dtype == VELORA_F32)
             z_to_bf16_kernel<float><<<static_cast<int>(grid), 256, 0, stream>>>(
                 static_cast<const float*>(Z), ldz, N, p.M, p.pitch, Zb);
+        else if (z_dtype == VELORA_FP8_E4M3)                  // every E4M3 value is a bf16 value: exact
+            z_to_bf16_kernel<e4m3_t><<<static_cast<int>(grid), 256, 0, stream>>>(
+                static_cast<const e4m3_t*>(Z), ldz, N, p.M, p.pitch, Zb);
         else
             z_to_bf16_kernel<__nv_bfloat16><<<static_cast<int>(grid), 256, 0, stream>>>(
                 static_cast<const __nv_bfloat16*>(Z), ldz, N, p.M, p.pitch, Zb);

@@ -80,6 +80,25 @@ def test_validation_happens_on_the_host_before_any_launch(lib):
     assert h(*args, 0, 5, good, 1 << 30, null) == b.ERR_INVALID_ARG                             # mode
     assert h(*args, 0, b.WG_FACTORED, null, 0, null) == b.ERR_WORKSPACE
     assert h(*args, 0, b.WG_FACTORED, good, 8, null) == b.ERR_WORKSPACE
+    # an empty batch may come with NULL data pointers: dW = beta * dW, nothing to launch when beta = 1
+    assert h(null, b.BF16, 0, 8, 8, null, b.F32, 4, null, 64, 16, good, b.BF16, 64, 1, b.WG_FACTORED,
+             good, 1 << 30, null) == b.OK
+    assert h(null, b.BF16, 0, 8, 8, null, b.F32, 4, null, 64, 16, null, b.BF16, 64, 1, b.WG_FACTORED,
+             good, 1 << 30, null) == b.ERR_INVALID_ARG                                          # dW is still needed
+    # the wait self-test validates its limit and workspace before launching
+    st = lib.velora_selftest_wait_timeout
+    assert st(good, 256, 10, good, null) == b.ERR_INVALID_ARG                                   # below 1 us
+    assert st(good, 256, 10 ** 9, good, null) == b.ERR_INVALID_ARG                              # above 100 ms
+    assert st(null, 256, 10 ** 6, good, null) == b.ERR_WORKSPACE
+    assert st(good, 256, 10 ** 6, null, null) == b.ERR_INVALID_ARG
+    # the 8-bit type is a storage type for Z only
+    assert f(good, b.FP8_E4M3, 4, 64, 64, 16, good, good, b.F32, 4, null) == b.ERR_UNSUPPORTED  # X in E4M3: no
+    assert h(good, b.BF16, 4, 8, 8, good, b.FP8_E4M3, 4, good, 64, 16, good, b.FP8_E4M3, 64, 0, b.WG_FACTORED,
+             good, 1 << 30, null) == b.ERR_UNSUPPORTED                                           # dW in E4M3: no
+    zc = lib.velora_z8_calibrate
+    assert zc(good, b.BF16, 4, 64, 64, 16, good, 0.5, good, good, good, good, 1 << 20, null) == b.ERR_INVALID_ARG   # headroom < 1
+    assert zc(good, b.BF16, 4, 64, 64, 16, good, 2.0, good, good, good, good, 16, null) == b.ERR_WORKSPACE
+    assert lib.velora_workspace_bytes(b.OP_Z8_CALIBRATE, 100, 64, 0, 16) >= 100 * 4 * 4
     # reconstruct / linear
     r = lib.velora_reconstruct
     assert r(good, b.F32, 4, 4, 64, 16, good, good, b.BF16, 60, null) == b.ERR_INVALID_ARG
@@ -116,3 +135,7 @@ def test_memory_model_matches_table_5b_structure():
     np.testing.assert_allclose(model, model[-1] + slope * (k - k[-1]), rtol=1e-12)
     assert saved_activation_bytes(N, D, 64) * 30 < saved_activation_bytes(N, D, None)
     assert saved_activation_bytes(10, 1376, 64) == 10 * 22 * 4 + 64 * 4      # ragged: ceil(1376/64) = 22
+    # storage types of Z: 4, 2 and 1 bytes per scalar; against the bf16 input at Dsub = 64 that is 32x, 64x, 128x
+    full = saved_activation_bytes(1 << 20, D, None)
+    for zb, ratio in ((4, 32), (2, 64), (1, 128)):
+        assert abs(full / saved_activation_bytes(1 << 20, D, 64, z_bytes=zb) / ratio - 1) < 1e-3

@@ -345,3 +345,71 @@ def test_generator_is_seeded_and_rounds_once():
     assert c1.dtype == "f32" and c1.shape == (256, 64)
     t = a.torch()
     assert t.shape == (64, 512) and np.array_equal(t.view(__import__("torch").int16).numpy().view(np.uint16), a.bits)
+
+
+# ------------------------------------------------------------------ E4M3 rounding helper (8-bit Z storage)
+def _e4m3_table():
+    """All finite E4M3 values straight from the format's definition: sign, exponent field E (bias 7),
+    mantissa field m; E = 0 is subnormal (m/8 * 2^-6); E = 15, m = 7 is NaN; there are no infinities."""
+    vals = []
+    for code in range(256):
+        s, E, m = code >> 7, (code >> 3) & 15, code & 7
+        if E == 15 and m == 7:
+            continue
+        mag = (m / 8.0) * 2.0 ** -6 if E == 0 else (1.0 + m / 8.0) * 2.0 ** (E - 7)
+        vals.append((code, -mag if s else mag))
+    return vals
+
+
+def test_round_to_fp8_e4m3_against_the_format_definition():
+    table = _e4m3_table()
+    assert len(table) == 254
+    vals = np.array([v for _, v in table])
+    assert vals.max() == 448.0 and np.min(np.abs(vals[vals != 0])) == 2.0 ** -9
+    # every representable value is a fixed point
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(vals), vals)
+    pos = np.array(sorted(v for c, v in table if c < 128))            # 0 .. 448, 127 values
+    codes = np.array(sorted(c for c, v in table if c < 128))
+    lo, hi = pos[:-1], pos[1:]
+    mid = 0.5 * (lo + hi)
+    # just below / above a midpoint goes to the nearer neighbour; the midpoint itself to the even code
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(mid * (1 - 1e-12)), lo)
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(mid * (1 + 1e-12)), hi)
+    even = np.where(codes[:-1] % 2 == 0, lo, hi)
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(mid), even)
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(-mid), -even)
+    # saturation, tiny values, specials
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3([449.0, 464.0, 1e9, -1e9, np.inf, -np.inf]),
+                                  [448.0, 448.0, 448.0, -448.0, 448.0, -448.0])
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3([2.0 ** -10, 2.0 ** -10 * 1.01, 2.0 ** -11]), [0.0, 2.0 ** -9, 0.0])
+    assert np.isnan(oracle.round_to_fp8_e4m3(np.nan))
+
+
+def test_round_to_fp8_e4m3_against_a_library_conversion():
+    """torch's float8_e4m3fn cast is an independent implementation of the same rounding (inside the
+    finite range; it does not saturate, so values are kept within +-448)."""
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.uniform(-448, 448, 20000), rng.standard_normal(20000) * 3,
+                        rng.standard_normal(20000) * 0.01, rng.uniform(-2.0 ** -5, 2.0 ** -5, 20000)]).astype(np.float32)
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    np.testing.assert_array_equal(oracle.round_to_fp8_e4m3(x.astype(np.float64)), lib)
+
+
+def test_fp8_z_store_scale_and_error_bound():
+    rng = np.random.default_rng(6)
+    Z = rng.standard_normal((300, 24)) * np.exp(rng.standard_normal(24))[None, :]
+    scale = oracle.zscale_from_batch(Z, headroom=2.0)
+    assert abs(scale * 448.0 - 2.0 * np.abs(Z).max()) < 1e-12
+    q = oracle.quantize_z_fp8(Z, scale)
+    assert np.abs(q).max() <= 448.0 / 2 + 16                      # headroom 2: the batch's own maximum sits at 224
+    deq = q * scale
+    normal = np.abs(Z) >= scale * 2.0 ** -6
+    assert np.all(np.abs(deq - Z)[normal] <= np.abs(Z)[normal] * 2.0 ** -4)      # half a unit of a 4-bit significand
+    assert np.all(np.abs(deq - Z)[~normal] <= scale * 2.0 ** -10)                # half the subnormal spacing
+    assert oracle.zscale_from_batch(np.zeros((3, 3))) == 1.0
+    assert oracle.zscale_from_batch(np.array([[np.nan]])) == 1.0
+    # a later batch that exceeds the calibrated range saturates instead of overflowing
+    assert oracle.quantize_z_fp8(np.array([1e6 * scale]), scale)[0] == 448.0
