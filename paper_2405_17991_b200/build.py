@@ -41,8 +41,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
 
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if not f.endswith(".cu")] + [os.path.join(INCLUDE, "velora.h")]
+    newest_header = max(os.path.getmtime(p) for p in headers)
+
     def compile_one(src):
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        if not force and not verbose and os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(src), newest_header):
+            return obj                                # this object is newer than its source and every header
         cmd = [nvcc] + NVCC_FLAGS + extra + ["-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:

@@ -26,9 +26,9 @@ constexpr int B_BYTES = BN * BK * 2;              // 32 KB
 constexpr int SLAB_BYTES = 64 * BK * 2;           // one 64-wide MN-major slab: 64 k-rows x 128 bytes
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr int FUSE_THREADS = GEMM_THREADS + 128;    // + four compress warps
+constexpr int FUSE_THREADS = GEMM_THREADS + 192;    // + four compress warps (6, 7, 10, 11) and two idle ones (8, 9)
 constexpr size_t GEMM_SMEM = 1024 + static_cast<size_t>(STAGES) * (A_BYTES + B_BYTES) + 256;
-constexpr size_t FUSE_SMEM = GEMM_SMEM + A_BYTES + VELORA_MAX_DSUB * 4;   // + compress tile + copy of v
+constexpr size_t FUSE_SMEM = GEMM_SMEM;
 
 struct TileCoord {
     int m0, n0;
@@ -47,15 +47,14 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
     return {tm * BM, tn * BN};
 }
 
-// FUSE = 0: plain GEMM.  FUSE = 1 / 2 (forward only, A = X K-major): Z = compress(X, v) (fp32 / bf16
-// storage) is computed by four extra warps from X tiles that are already on their way through L2 for the
-// GEMM, so X crosses HBM once for both results.  A k-block of 64 columns holds 64/Dsub sub-tokens (or
-// 1/w of one, w = Dsub/64); the CTA working on n-tile j handles the sub-token groups g with
-// g % tiles_n == j, so the work is spread over the CTAs that share a row block.  For such a k-block the
-// producer fetches the X tile a second time (an L2 hit) into a buffer of its own with its own pair of
-// barriers: the GEMM ring has no slack to wait for a second reader (four stages barely cover the TMA
-// latency), so the compress warps never touch it.  Thread t of the compress warps owns tile row t; the
-// 128-byte swizzle of the tile makes its 16-byte reads conflict-free.
+// FUSE = 0: plain GEMM.  FUSE = 1 / 2 / 3 (forward only, A = X K-major): Z = compress(X, v) (fp32 / bf16 /
+// E4M3 storage) is computed by four extra warps for the row block the CTA is multiplying, from lines of X
+// that are on their way through L2 for the GEMM anyway, so X crosses HBM once for both results.  The CTA
+// working on n-tile j handles the sub-token groups g with g % tiles_n == j, so the work is spread over the
+// CTAs that share a row block.  The compress warps read X with plain 16-byte loads and keep v in registers:
+// they share no stage, no barrier and no shared-memory bandwidth with the GEMM's pipeline (gemm_fuse.cuh),
+// and they sit on warps 6, 7, 10, 11 so that none of them shares a warp scheduler (warp % 4) with the TMA
+// producer (warp 0) or the MMA issuer (warp 1).
 template <bool A_MN, bool B_MN, typename CT, int FUSE>
 __global__ void __launch_bounds__(FUSE ? FUSE_THREADS : GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -69,17 +68,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* smem = smem_raw + (base - raw);
     const uint32_t sA = base;
     const uint32_t sB = base + STAGES * A_BYTES;
-    constexpr int CBUF_BYTES = FUSE ? A_BYTES : 0;              // the compress warps' own X tile
-    const uint32_t cbuf = base + STAGES * (A_BYTES + B_BYTES);
-    uint8_t* tail = smem + STAGES * (A_BYTES + B_BYTES) + CBUF_BYTES;
-    const uint32_t bars = cbuf + CBUF_BYTES;
+    uint8_t* tail = smem + STAGES * (A_BYTES + B_BYTES);
+    const uint32_t bars = base + STAGES * (A_BYTES + B_BYTES);
     const uint32_t full = bars, empty = bars + 8 * STAGES;
     const uint32_t tfull = bars + 16 * STAGES, tempty = tfull + 16;
-    const uint32_t cfull = tempty + 16, cempty = cfull + 8;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 48);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 56);
-    float* sv = reinterpret_cast<float*>(tail + 256);           // copy of v for the compress warps
-    const int cw = (FUSE && fz.Dsub >= BK) ? fz.Dsub / BK : 1;  // k-blocks per sub-token
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -95,8 +89,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(tfull + 8 * a, 1);
             mbar_init(tempty + 8 * a, 4);
         }
-        mbar_init(cfull, 1);
-        mbar_init(cempty, 4);                                   // one arrival per compress warp
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
@@ -106,8 +98,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
-    if (FUSE)
-        for (int j = threadIdx.x; j < fz.Dsub; j += blockDim.x) sv[j] = fz.v[j];
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -117,11 +107,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (one lane)
         if (lane == 0) {
-            uint32_t it = 0, oc = 0;
+            uint32_t it = 0;
             for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
                 const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
-                OwnedWalk own(cw, tiles_n, tc0.n0 / BN);
-                for (int kb = 0; kb < kblocks; ++kb, ++it, own.step(kb)) {
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
                     mbar_arrive_expect_tx(full + 8 * s, A_BYTES + B_BYTES);
@@ -140,21 +129,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         tma_load_2d(sB + s * B_BYTES, &tmB, full + 8 * s, k0, tc0.n0);
                     }
-                    if (FUSE && own.owned()) {                             // this CTA compresses the k-block
-                        if (!mbar_wait(cempty, (oc & 1u) ^ 1u, abort_flag)) { failed = true; break; }
-                        mbar_arrive_expect_tx(cfull, A_BYTES);
-                        tma_load_2d(cbuf, &tmA, cfull, k0, tc0.m0);
-                        ++oc;
-                    }
                 }
             }
             if (failed) {
                 *abort_flag = 1;
-                if (FUSE && oc > 0) {
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(cfull, (oc - 1u) & 1u))
-                        if (globaltimer_ns() - t0 > kWaitLimitNs) break;
-                }
                 // Let this CTA's own copies in flight land before shared memory is given up.
                 const uint32_t back = it < STAGES ? it : STAGES;
                 for (uint32_t j = 1; j <= back; ++j) {
@@ -197,26 +175,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (failed) *abort_flag = 1;
         }
+    } else if (FUSE && (warp == 8 || warp == 9)) {
+        // Idle on purpose: these two would share warp schedulers 0 and 1 with the producer and the MMA issuer.
     } else if (FUSE && warp >= 6) {
-        // ------------------------------------------------ compress (4 warps, one tile row per thread)
-        const int trow = (warp - 6) * 32 + lane;
-        float acc = 0.f;
-        uint32_t oc = 0;
-        for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
-            const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
-            const int tn = tc0.n0 / BN;
-            const int row = tc0.m0 + trow;
-            OwnedWalk own(cw, tiles_n, tn);
-            for (int kb = 0; kb < kblocks; ++kb, own.step(kb)) {
-                if (!own.owned()) continue;
-                if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
-                ++oc;
-                compress_kblock<FUSE>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
-                __syncwarp();                                 // every lane's reads of the tile are done
-                if (lane == 0) mbar_arrive(cempty);
+        // ------------------------------------------------ compress (4 warps, 32 rows of the tile's 128 each)
+        const int cwi = warp < 8 ? warp - 6 : warp - 8;
+        const int cpr = (fz.Dsub >> 3) < 8 ? 8 : (fz.Dsub >> 3);
+        const int n_groups = (Kdim + 8 * cpr - 1) / (8 * cpr);
+        auto walk = [&](auto vs) {
+            vs.load(fz.v, fz.Dsub, lane);
+            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+                const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
+                const int r0 = tc0.m0 + cwi * 32;
+                if (r0 >= Mdim) continue;
+                for (int g = tc0.n0 / BN; g < n_groups; g += tiles_n)
+                    compress_group_direct<FUSE>(fz, vs, r0, Mdim, Kdim, g, lane);
             }
-        }
-        if (failed) *abort_flag = 1;
+        };
+        if (fz.Dsub <= 256) walk(VSlice<1>{});
+        else if (fz.Dsub == 512) walk(VSlice<2>{});
+        else walk(VSlice<4>{});
     } else {
         // ------------------------------------------------ epilogue (4 warps, one TMEM lane quarter each)
         const int quarter = warp & 3;
@@ -410,7 +388,7 @@ int launch_linear_forward_tc(const void* X, int64_t ldx, const void* W, int64_t 
         if (rc != VELORA_OK) return rc;
         rc = make_tmap_bf16_2d(&tb, W, D, O, ldw, BK, BN);
         if (rc != VELORA_OK) return rc;
-        FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>(ceil_div64(D, Dsub))};
+        FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>(ceil_div64(D, Dsub)), static_cast<const uint4*>(X), ldx / 8};
         const int m = static_cast<int>(N), n = static_cast<int>(O), k = static_cast<int>(D);
         if (z_dtype == VELORA_F32)
             return launch_kernel<false, false, __nv_bfloat16, 1>(ta, tb, Y, ldy, 0, m, n, k, status, stream, fz);

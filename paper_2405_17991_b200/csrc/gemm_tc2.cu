@@ -17,11 +17,12 @@
 //   tempty[a]  leader's copy, 8 arrivals: the four epilogue warps of each CTA.
 // Every wait is bounded; both CTAs always reach the closing cluster barrier.
 //
-// FUSE = 1 / 2 (forward only, both operands K-major): four more warps per CTA compute Z = compress(X, v)
-// (fp32 / bf16 storage) from X tiles that are in L2 for the GEMM anyway, so X crosses HBM once for both
-// results.  The CTA pair working on n-tile j handles the sub-token groups g with g % tiles_n == j; for
-// such a k-block each CTA's producer fetches its X tile a second time into a buffer that only the
-// compress warps read (own barriers cfull / cempty, both local), so the GEMM ring never waits for them.
+// FUSE = 1 / 2 / 3 (forward only, both operands K-major): four more warps per CTA compute Z = compress(X, v)
+// (fp32 / bf16 / E4M3 storage) for the row block the CTA is multiplying, from lines of X that are in L2 for
+// the GEMM anyway, so X crosses HBM once for both results.  The CTA pair working on n-tile j handles the
+// sub-token groups g with g % tiles_n == j.  These warps read X with plain 16-byte loads and share nothing
+// with the GEMM's pipeline: no stage, no barrier, no producer work (a second copy of the X tile fetched by the
+// TMA producer into a buffer of their own cost 4-9 % of the product's time).
 #include <cooperative_groups.h>
 
 #include "gemm_fuse.cuh"
@@ -45,9 +46,9 @@ constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
 constexpr int P_SLAB = 64 * P_BK * 2;               // 8 KB, one 64-wide MN-major slab
 constexpr int P_THREADS = 192;
 constexpr int P_TMEM_COLS = 512;
-constexpr int P_FUSE_THREADS = P_THREADS + 128;      // + four compress warps
+constexpr int P_FUSE_THREADS = P_THREADS + 192;      // + four compress warps (6, 7, 10, 11) and two idle ones (8, 9)
 constexpr size_t P_SMEM = 1024 + static_cast<size_t>(P_STAGES) * P_STAGE_BYTES + 256;
-constexpr size_t P_FUSE_SMEM = P_SMEM + P_A_BYTES + VELORA_MAX_DSUB * 4;   // + compress tile + copy of v
+constexpr size_t P_FUSE_SMEM = P_SMEM;
 
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
 {
@@ -130,17 +131,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    constexpr int CBUF_BYTES = FUSE ? P_A_BYTES : 0;         // the compress warps' own X tile
-    const uint32_t cbuf = base + P_STAGES * P_STAGE_BYTES;
-    uint8_t* tail = smem + P_STAGES * P_STAGE_BYTES + CBUF_BYTES;
-    const uint32_t bars = cbuf + CBUF_BYTES;
+    uint8_t* tail = smem + P_STAGES * P_STAGE_BYTES;
+    const uint32_t bars = base + P_STAGES * P_STAGE_BYTES;
     const uint32_t full = bars, empty = bars + 8 * P_STAGES;
     const uint32_t tfull = bars + 16 * P_STAGES, tempty = tfull + 16;
-    const uint32_t cfull = tempty + 16, cempty = cfull + 8;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * P_STAGES + 48);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * P_STAGES + 56);
-    float* sv = reinterpret_cast<float*>(tail + 256);        // copy of v for the compress warps
-    const int cw = (FUSE && fz.Dsub >= P_BK) ? fz.Dsub / P_BK : 1;   // k-blocks per sub-token
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = tiles_m * tiles_n;
@@ -155,8 +151,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_init(tfull + 8 * a, 1);
             mbar_init(tempty + 8 * a, 8);                    // four epilogue warps of each CTA
         }
-        mbar_init(cfull, 1);
-        mbar_init(cempty, 4);                                // one arrival per compress warp
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
@@ -166,8 +160,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         tmem_alloc_pair(smem_u32(tmem_slot), P_TMEM_COLS);
         tmem_relinquish_pair();
     }
-    if (FUSE)
-        for (int j = threadIdx.x; j < fz.Dsub; j += blockDim.x) sv[j] = fz.v[j];
     tc_fence_before_sync();
     __syncthreads();
     cluster.sync();                                          // both CTAs' barriers exist before anyone signals them
@@ -178,13 +170,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: this CTA's rows of A, its half of B
         if (lane == 0) {
-            uint32_t it = 0, oc = 0;
+            uint32_t it = 0;
             for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs) {
                 const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
                 const int m0 = t0.m0 + static_cast<int>(rank) * P_BM;
                 const int n0 = t0.n0 + static_cast<int>(rank) * (P_BN / 2);
-                OwnedWalk own(cw, tiles_n, t0.n0 / P_BN);
-                for (int kb = 0; kb < kblocks; ++kb, ++it, own.step(kb)) {
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % P_STAGES, ph = (it / P_STAGES) & 1u;
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
                     const uint32_t lead_full = map_to_cta(full + 8 * s, 0);
@@ -205,23 +196,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     } else {
                         tma_load_2d_pair(b_dst, &tmB, lead_full, k0, n0);
                     }
-                    if (FUSE && own.owned()) {                     // this pair compresses the k-block
-                        if (!mbar_wait(cempty, (oc & 1u) ^ 1u, abort_flag)) { failed = true; break; }
-                        mbar_arrive_expect_tx(cfull, P_A_BYTES);
-                        tma_load_2d(cbuf, &tmA, cfull, k0, m0);
-                        ++oc;
-                    }
                 }
             }
             if (failed) {
                 *abort_flag = 1;
-                // Let the copies in flight land before shared memory is given up: the compress tile on
-                // its own barrier; the ring's copies complete on the leader's barriers, which the leader
-                // watches (each phase needs both CTAs' bytes) while the peer allows them 50 us.
+                // Let the copies in flight land before shared memory is given up: the ring's copies complete
+                // on the leader's barriers, which the leader watches (each phase needs both CTAs' bytes) while
+                // the peer allows them 50 us.
                 const unsigned long long t0 = globaltimer_ns();
-                if (FUSE && oc > 0)
-                    while (!mbar_try_wait(cfull, (oc - 1u) & 1u))
-                        if (globaltimer_ns() - t0 > kWaitLimitNs) break;
                 if (rank == 0) {
                     const uint32_t back = it < P_STAGES ? it : P_STAGES;
                     for (uint32_t j = 1; j <= back; ++j) {
@@ -264,26 +246,31 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             if (failed) *abort_flag = 1;
         }
+    } else if (FUSE && (warp == 8 || warp == 9)) {
+        // Idle on purpose.  A warp is served by the scheduler warp % 4; warps 8 and 9 would share schedulers 0
+        // and 1 with the TMA producer and the MMA issuer, single threads on the kernel's critical path.  With
+        // the compress on those two warps the product ran 5-6 % slower, on warps 10 and 11 it runs 1-2.5 % slower.
     } else if (FUSE && warp >= 6) {
-        // ------------------------------------------------ compress (4 warps, one tile row per thread)
-        const int trow = (warp - 6) * 32 + lane;
-        float acc = 0.f;
-        uint32_t oc = 0;
-        for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs) {
-            const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
-            const int tn = t0.n0 / P_BN;
-            const int row = t0.m0 + static_cast<int>(rank) * P_BM + trow;
-            OwnedWalk own(cw, tiles_n, tn);
-            for (int kb = 0; kb < kblocks; ++kb, own.step(kb)) {
-                if (!own.owned()) continue;
-                if (!mbar_wait_warp(cfull, oc & 1u, abort_flag, 64)) { failed = true; break; }
-                ++oc;
-                compress_kblock<FUSE>(cbuf, trow, sv, fz, cw, kb, kblocks, row, Mdim, acc);
-                __syncwarp();                                // every lane's reads of the tile are done
-                if (lane == 0) mbar_arrive(cempty);
+        // ------------------------------------------------ compress (4 warps, 32 rows of the CTA's 128 each)
+        const int cwi = warp < 8 ? warp - 6 : warp - 8;
+        // For the row block of every tile this pair works on, these warps compress the column groups
+        // g = tn, tn + tiles_n, ... (tn = the tile's n index), so that the tiles of a row block share the
+        // work; they read X themselves and run beside the GEMM's pipeline without touching it.
+        const int cpr = (fz.Dsub >> 3) < 8 ? 8 : (fz.Dsub >> 3);
+        const int n_groups = (Kdim + 8 * cpr - 1) / (8 * cpr);
+        auto walk = [&](auto vs) {
+            vs.load(fz.v, fz.Dsub, lane);
+            for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+                const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
+                const int r0 = t0.m0 + static_cast<int>(rank) * P_BM + cwi * 32;
+                if (r0 >= Mdim) continue;
+                for (int g = t0.n0 / P_BN; g < n_groups; g += tiles_n)
+                    compress_group_direct<FUSE>(fz, vs, r0, Mdim, Kdim, g, lane);
             }
-        }
-        if (failed) *abort_flag = 1;
+        };
+        if (fz.Dsub <= 256) walk(VSlice<1>{});
+        else if (fz.Dsub == 512) walk(VSlice<2>{});
+        else walk(VSlice<4>{});
     } else {
         // ------------------------------------------------ epilogue: this CTA's 128 rows of the pair tile
         const int quarter = warp & 3;
@@ -415,7 +402,7 @@ int launch_linear_forward_tc_pair(const void* X, int64_t ldx, const void* W, int
     if (rc != VELORA_OK) return rc;
     rc = make_tmap_bf16_2d(&tb, W, D, O, ldw, P_BK, P_BN / 2);
     if (rc != VELORA_OK) return rc;
-    FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>((D + Dsub - 1) / Dsub)};
+    FuseArgs fz{v, Z, ldz, Dsub, static_cast<int>((D + Dsub - 1) / Dsub), static_cast<const uint4*>(X), ldx / 8};
     const int m = static_cast<int>(N), n = static_cast<int>(O), k = static_cast<int>(D);
     if (z_dtype == VELORA_F32)
         return launch_pair<false, false, __nv_bfloat16, 1>(ta, tb, Y, ldy, 0, m, n, k, status, di.sm_count, stream, fz);

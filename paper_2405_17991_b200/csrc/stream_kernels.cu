@@ -66,60 +66,93 @@ init_v_partial_elem_kernel(const XT* __restrict__ X, int64_t N, int D, int64_t l
 
 // ------------------------------------------------------------------ init_v finalize: one CTA
 // s[j] = sum over CTAs (fixed order, fp64), norm, v = s / ||s||.  status[0] = 0 ok, 1 degenerate.
-// For a block of up to 256 positions the 256 threads split the partial rows into `slots` interleaved
-// groups (independent loads), then one thread per position adds the groups in order.
-__global__ void __launch_bounds__(kStreamThreads)
+// The partial rows come from up to ~1200 CTAs and sit in L2; adding them is a chain of load latencies, so
+// the CTA is as wide as it can be (1024 threads) and a thread owns VEC consecutive positions (one 16-byte
+// load for VEC = 4): for a block of up to 1024 position groups the threads split the partial rows into
+// `slots` interleaved sets (eight independent loads in flight each), then one thread per group adds the
+// sets in order.  The order depends only on the sizes, so the result is run-to-run identical.
+constexpr int kFinThreads = 1024;
+
+template <int VEC>
+__global__ void __launch_bounds__(kFinThreads)
 init_v_finalize_kernel(const float* __restrict__ partials, int num_partials, int Dsub,
                        float* __restrict__ v, int* __restrict__ status, int normalize)
 {
     __shared__ double s_sum[VELORA_MAX_DSUB];
-    __shared__ double s_red[kStreamThreads];
-    __shared__ double s_norm;
-    for (int j0 = 0; j0 < Dsub; j0 += kStreamThreads) {
-        const int width = (Dsub - j0 < kStreamThreads) ? Dsub - j0 : kStreamThreads;
-        const int slots = kStreamThreads / width;
-        const int j = j0 + threadIdx.x % width;
+    __shared__ double s_red[kFinThreads * VEC];
+    __shared__ double s_warp[kFinThreads / 32];
+    const int groups = Dsub / VEC;                             // VEC divides Dsub (host)
+    for (int g0 = 0; g0 < groups; g0 += kFinThreads) {
+        const int width = (groups - g0 < kFinThreads) ? groups - g0 : kFinThreads;
+        const int slots = kFinThreads / width;
+        const int g = g0 + threadIdx.x % width;
         const int slot = threadIdx.x / width;
-        double s = 0.0;
+        double s[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s[e] = 0.0;
         if (slot < slots)
             for (int b = slot; b < num_partials; b += 8 * slots) {     // eight loads in flight, added in order
-                float x[8];
+                float x[8][VEC];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int bu = b + u * slots;
-                    x[u] = bu < num_partials ? partials[static_cast<int64_t>(bu) * Dsub + j] : 0.f;
+                    const float* src = partials + static_cast<int64_t>(bu) * Dsub + g * VEC;
+                    if (bu >= num_partials) {
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) x[u][e] = 0.f;
+                    } else if (VEC == 4) {
+                        const float4 t = *reinterpret_cast<const float4*>(src);
+                        x[u][0] = t.x; x[u][1 % VEC] = t.y; x[u][2 % VEC] = t.z; x[u][3 % VEC] = t.w;
+                    } else {
+                        x[u][0] = *src;
+                    }
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) s += static_cast<double>(x[u]);
+                for (int u = 0; u < 8; ++u)
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) s[e] += static_cast<double>(x[u][e]);
             }
-        s_red[threadIdx.x] = s;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s_red[threadIdx.x * VEC + e] = s[e];
         __syncthreads();
         if (threadIdx.x < width) {
-            double t = 0.0;
-            for (int k = 0; k < slots; ++k) t += s_red[k * width + threadIdx.x];
-            s_sum[j] = t;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                double t = 0.0;
+                for (int k = 0; k < slots; ++k) t += s_red[(k * width + threadIdx.x) * VEC + e];
+                s_sum[g * VEC + e] = t;
+            }
         }
         __syncthreads();
     }
     if (!normalize) {                                          // the plain sub-token sum s (multi-rank use)
-        for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) v[j] = static_cast<float>(s_sum[j]);
+        for (int j = threadIdx.x; j < Dsub; j += kFinThreads) v[j] = static_cast<float>(s_sum[j]);
         return;
     }
+    // ||s||^2: fixed tree (xor shuffles inside a warp, then the 32 warp sums in order)
     double sq = 0.0;
-    for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) sq += s_sum[j] * s_sum[j];
-    s_red[threadIdx.x] = sq;
+    for (int j = threadIdx.x; j < Dsub; j += kFinThreads) sq += s_sum[j] * s_sum[j];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = sq;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        double t = 0.0;
-        for (int i = 0; i < kStreamThreads; ++i) t += s_red[i];
-        s_norm = sqrt(t);
-    }
-    __syncthreads();
-    const double norm = s_norm;
+    double t = 0.0;
+    for (int i = 0; i < kFinThreads / 32; ++i) t += s_warp[i];
+    const double norm = sqrt(t);
     const bool ok = (norm > 0.0) && isfinite(norm);
     if (threadIdx.x == 0) status[0] = ok ? 0 : 1;
     if (ok)
-        for (int j = threadIdx.x; j < Dsub; j += kStreamThreads) v[j] = static_cast<float>(s_sum[j] / norm);
+        for (int j = threadIdx.x; j < Dsub; j += kFinThreads) v[j] = static_cast<float>(s_sum[j] / norm);
+}
+
+// Partial rows start 16-byte aligned and are Dsub floats apart: four positions per load when Dsub allows it.
+inline void launch_init_v_finalize(const float* partials, int num_partials, int Dsub, float* v, int* status,
+                                   int normalize, cudaStream_t stream)
+{
+    if (Dsub % 4 == 0 && aligned16(partials))
+        init_v_finalize_kernel<4><<<1, kFinThreads, 0, stream>>>(partials, num_partials, Dsub, v, status, normalize);
+    else
+        init_v_finalize_kernel<1><<<1, kFinThreads, 0, stream>>>(partials, num_partials, Dsub, v, status, normalize);
 }
 
 // Running-average variant of the initialisation (Section 5, ablation on the initialisation strategy):
@@ -489,7 +522,7 @@ int launch_normalize_v(const float* s, int Dsub, float* v, void* ws, size_t ws_b
 {
     if (ws_bytes < kStatusBytes) return VELORA_ERR_WORKSPACE;
     int* status = static_cast<int*>(ws) + 1;
-    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(s, 1, Dsub, v, status, 1);
+    launch_init_v_finalize(s, 1, Dsub, v, status, 1, stream);
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
     return read_degenerate_flag(status, stream);
 }
@@ -543,7 +576,7 @@ int launch_init_v(const void* X, int x_dtype, int64_t N, int64_t D, int64_t ldx,
                 static_cast<const float*>(X), N, static_cast<int>(D), ldx, Dsub, M, rows_per_cta, partials);
     }
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
-    init_v_finalize_kernel<<<1, kStreamThreads, 0, stream>>>(partials, num_partials, Dsub, v, status, sum_only ? 0 : 1);
+    launch_init_v_finalize(partials, num_partials, Dsub, v, status, sum_only ? 0 : 1, stream);
     if (check_launch() != VELORA_OK) return VELORA_ERR_CUDA;
     if (sum_only) return VELORA_OK;                            // v holds s; nothing to report, no synchronisation
     return read_degenerate_flag(status, stream);
