@@ -400,12 +400,20 @@ def run_ours(args):
                     row = {"shape": r["shape"], "Dsub": r["Dsub"], "bytes": r["bytes"], "us": r["us"], "GB/s": r["GB/s"],
                            "frac": r["frac_measured"], "frac_nominal_8TBs": r["GB/s"] / NOMINAL_HBM_GBS}
                     for k_src, k_dst in (("us_back_to_back", "us_back_to_back"), ("frac_measured_back_to_back", "frac_back_to_back"),
+                                         ("us_graph", "us_graph"), ("frac_measured_graph", "frac_graph"),
                                          ("TFLOP/s", "TFLOP/s"), ("roofline_TFLOP/s", "roofline_TFLOP/s")):
                         if k_src in r:
                             row[k_dst] = r[k_src]
                     rows.append(row)
             return rows
         line["roofline"]["hbm_peak_GB/s"] = pk["hbm_gbs"]
+        floor = line["kernels"][0]
+        line["roofline"]["timing_floor_us"] = {
+            "per_call": floor["us"], "back_to_back": floor["us_back_to_back"], "graph": floor["us_graph"],
+            "note": "device time of the smallest compress (one CTA) timed the same three ways: `us` = one call between its own "
+                    "pair of CUDA events, `us_back_to_back` = calls queued behind one another inside one pair of events, "
+                    "`us_graph` = the same calls replayed from a CUDA graph. A kernel of 10-30 us cannot show more than "
+                    "t_min / (t_min + per_call floor) in the per-call column."}
         line["roofline"]["compress"] = pick("compress")
         line["roofline"]["reconstruct"] = pick("reconstruct")
         line["roofline"]["weight_grad_factored"] = pick("weight_grad factored")
@@ -528,7 +536,34 @@ def kernel_table(vl, torch, L, N, ws, pk):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / (reps * len(fn_list))
 
-    def hbm(name, shape, ms, nbytes, ms_b2b=None, dsub=DSUB):
+    def timed_graph(fn_list, rounds=5, reps=5):
+        """Device time per call (ms) when rounds x len(fn_list) calls are captured once into a CUDA graph and
+        the graph is replayed: no host submission at all between the kernels, so this is what a call costs the
+        GPU inside a captured step (kernel, launch gap and drain), free of the event pair's own latency and of
+        the host's submission rate, which bounds the back-to-back figure of the shortest kernels."""
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for f in fn_list:
+                f()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(rounds):
+                for f in fn_list:
+                    f()
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (rounds * reps * len(fn_list))
+
+    def hbm(name, shape, ms, nbytes, ms_b2b=None, dsub=DSUB, ms_graph=None):
         gbs = nbytes / (ms * 1e-3) / 1e9
         row = {"kernel": name, "shape": shape, "Dsub": dsub, "bytes": nbytes, "us": ms * 1e3, "GB/s": gbs, "bound": "hbm",
                "frac_measured": gbs / pk["hbm_gbs"], "frac_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
@@ -536,6 +571,9 @@ def kernel_table(vl, torch, L, N, ws, pk):
             g2 = nbytes / (ms_b2b * 1e-3) / 1e9
             row.update({"us_back_to_back": ms_b2b * 1e3, "GB/s_back_to_back": g2,
                         "frac_measured_back_to_back": g2 / pk["hbm_gbs"], "frac_nominal_8TBs_back_to_back": g2 / NOMINAL_HBM_GBS})
+        if ms_graph is not None:
+            g3 = nbytes / (ms_graph * 1e-3) / 1e9
+            row.update({"us_graph": ms_graph * 1e3, "GB/s_graph": g3, "frac_measured_graph": g3 / pk["hbm_gbs"]})
         out.append(row)
 
     def tensor(name, shape, ms, flops, nbytes=None, dsub=DSUB):
@@ -548,6 +586,15 @@ def kernel_table(vl, torch, L, N, ws, pk):
             row.update({"bound": "hbm", "bytes": nbytes, "GB/s": gbs, "frac_measured": gbs / pk["hbm_gbs"],
                         "roofline_TFLOP/s": min(pk["bf16_tflops"], ai * pk["hbm_gbs"] / 1e3)})
         out.append(row)
+
+    # What the three ways of timing cost by themselves: the smallest compress (8 tokens of 64 columns, one CTA).
+    tx = torch.zeros((8, 64), dtype=torch.bfloat16, device=dev)
+    tv = torch.ones(64, dtype=torch.float32, device=dev)
+    tz = torch.empty((8, 1), dtype=torch.float32, device=dev)
+    tiny = [lambda: vl.velora_compress(tx, tv, Z=tz)]
+    out.append({"kernel": "timing floor: compress of 8 tokens x 64 columns (one CTA)", "shape": "N=8 D=64", "Dsub": 64,
+                "bound": "latency", "us": timed(tiny, reps=21) * 1e3, "us_back_to_back": timed_b2b(tiny, reps=50) * 1e3,
+                "us_graph": timed_graph(tiny, rounds=20) * 1e3})
 
     # The second sub-token length of the configuration: its own v and Z per layer.
     for l in L:
@@ -564,15 +611,15 @@ def kernel_table(vl, torch, L, N, ws, pk):
         for group, label in ((small, "N=%d D=4096" % N), ([big], "N=%d D=11008" % N)):
             D, M = group[0]["D"], group[0][km]
             fns = [(lambda l=l: vl.velora_compress(l["X"], l[kv], Z=l[kz])) for l in group]
-            hbm("compress", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub)
+            hbm("compress", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub, timed_graph(fns))
             fns = [(lambda l=l: vl.velora_reconstruct(l[kz], l[kv], D, Xhat=l["dX"])) for l in group]
-            hbm("reconstruct", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub)
+            hbm("reconstruct", label, timed(fns), N * D * 2 + N * M * 4, timed_b2b(fns), dsub, timed_graph(fns))
             if dsub == DSUB:
                 ms = timed([(lambda l=l: vl.velora_init_v(l["X"], DSUB, v=l["v"], ws=ws)) for l in group])
                 hbm("init_v (incl. the stream sync that reads the degenerate flag)", label, ms, N * D * 2)
                 svec = torch.empty(DSUB, dtype=torch.float32, device=dev)
                 fns = [(lambda l=l: vl.velora_subtoken_sum(l["X"], DSUB, s=svec, ws=ws)) for l in group]
-                hbm("subtoken_sum (init_v's two kernels, no sync)", label, timed(fns), N * D * 2, timed_b2b(fns))
+                hbm("subtoken_sum (init_v's two kernels, no sync)", label, timed(fns), N * D * 2, timed_b2b(fns), DSUB, timed_graph(fns))
     # context only: torch's own fill and reduction on the same 180 MB buffer (pure write / pure read ceilings)
     big_x = big["dX"]
     hbm("reference: torch zero_ (pure write, library kernel)", "N=%d D=11008" % N, timed([lambda: big_x.zero_()]),
@@ -590,9 +637,24 @@ def kernel_table(vl, torch, L, N, ws, pk):
             fl = layer_flops(N, l0["D"], l0["O"], l0[km])["dw"]
             nb = N * l0["O"] * 2 + N * l0[km] * 4 + l0["O"] * l0["D"] * 2
             tensor("weight_grad factored", "%dx%d -> dW[%d,%d]" % (N, l0["O"], l0["O"], l0["D"]), ms, fl, nb, dsub)
-            ms2 = timed_b2b(fns)
+            ms2, ms3 = timed_b2b(fns), timed_graph(fns)
             out[-1].update({"us_back_to_back": ms2 * 1e3, "GB/s_back_to_back": nb / (ms2 * 1e-3) / 1e9,
-                            "frac_measured_back_to_back": nb / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"]})
+                            "frac_measured_back_to_back": nb / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"],
+                            "us_graph": ms3 * 1e3, "GB/s_graph": nb / (ms3 * 1e-3) / 1e9,
+                            "frac_measured_graph": nb / (ms3 * 1e-3) / 1e9 / pk["hbm_gbs"]})
+    # the same with Z stored in bf16 (read in place by the tensor map: no conversion launch)
+    for l in L:
+        l["Zb"] = l["Z"].to(torch.bfloat16)
+    for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
+        group = [by[n] for n in names]
+        l0 = group[0]
+        fns = [(lambda l=l: vl.velora_weight_grad(l["dY"], l["Zb"], l["v"], l["D"], dW=l["dW"], ws=ws)) for l in group]
+        fl = layer_flops(N, l0["D"], l0["O"], l0["M"])["dw"]
+        nb = N * l0["O"] * 2 + N * l0["M"] * 2 + l0["O"] * l0["D"] * 2
+        tensor("weight_grad factored, Z stored in bf16", "%dx%d -> dW[%d,%d]" % (N, l0["O"], l0["O"], l0["D"]), timed(fns), fl, nb)
+        ms2, ms3 = timed_b2b(fns), timed_graph(fns)
+        out[-1].update({"us_back_to_back": ms2 * 1e3, "frac_measured_back_to_back": nb / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"],
+                        "us_graph": ms3 * 1e3, "frac_measured_graph": nb / (ms3 * 1e-3) / 1e9 / pk["hbm_gbs"]})
     # dense contractions
     for names in (("q", "k", "v", "o"), ("up", "gate"), ("down",)):
         group = [by[n] for n in names]
