@@ -15,6 +15,29 @@ struct FuseArgs {
     int64_t ldx_chunks;
 };
 
+// The compress warps keep step with the GEMM: they take the row block of the CTA's ti-th tile only once the
+// TMA producer has started on that tile (it publishes the number of tiles started in shared memory), so their
+// loads of X meet the GEMM's in L2 instead of running a hundred microseconds ahead and sending X through HBM
+// a second time.  A hint, not a barrier: nothing waits for the compress warps.  Bounded like every wait: gives
+// up when another role has raised the abort flag or after a second.
+__device__ __forceinline__ bool wait_for_tile(volatile int* tiles_started, int ti, volatile int* abort_flag)
+{
+    if (*tiles_started > ti) return true;
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    unsigned spins = 0;
+    while (*tiles_started <= ti) {
+        __nanosleep(200);
+        if ((++spins & 15u) == 0u) {
+            if (*abort_flag) return false;
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+            if (t - t0 > 1000000000ull) return false;
+        }
+    }
+    return true;
+}
+
 template <int ZK> __device__ __forceinline__ void store_z(const FuseArgs& fz, int row, int m, float z)
 {
     if (ZK == 2) static_cast<__nv_bfloat16*>(fz.Z)[static_cast<int64_t>(row) * fz.ldz + m] = __float2bfloat16_rn(z);

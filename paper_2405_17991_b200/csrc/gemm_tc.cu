@@ -74,6 +74,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tfull = bars + 16 * STAGES, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * STAGES + 48);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 56);
+    volatile int* tiles_started = reinterpret_cast<volatile int*>(tail + 16 * STAGES + 60);   // producer's progress, read by the compress warps
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -90,6 +91,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(tempty + 8 * a, 4);
         }
         *abort_flag = 0;
+        *tiles_started = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
@@ -108,7 +110,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------ TMA producer (one lane)
         if (lane == 0) {
             uint32_t it = 0;
+            int started = 0;
             for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
+                if (FUSE) *tiles_started = ++started;          // the compress warps may take this tile's row block now
                 const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
@@ -184,7 +188,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int n_groups = (Kdim + 8 * cpr - 1) / (8 * cpr);
         auto walk = [&](auto vs) {
             vs.load(fz.v, fz.Dsub, lane);
-            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+            int ti = 0;
+            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++ti) {
+                if (!wait_for_tile(tiles_started, ti, abort_flag)) { failed = true; break; }
                 const TileCoord tc0 = tile_coord(tile, tiles_m, tiles_n);
                 const int r0 = tc0.m0 + cwi * 32;
                 if (r0 >= Mdim) continue;

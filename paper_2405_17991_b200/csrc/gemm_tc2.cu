@@ -137,6 +137,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tfull = bars + 16 * P_STAGES, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16 * P_STAGES + 48);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * P_STAGES + 56);
+    volatile int* tiles_started = reinterpret_cast<volatile int*>(tail + 16 * P_STAGES + 60);   // producer's progress, read by the compress warps
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = tiles_m * tiles_n;
@@ -152,6 +153,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_init(tempty + 8 * a, 8);                    // four epilogue warps of each CTA
         }
         *abort_flag = 0;
+        *tiles_started = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
@@ -171,7 +173,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------ TMA producer: this CTA's rows of A, its half of B
         if (lane == 0) {
             uint32_t it = 0;
+            int started = 0;
             for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs) {
+                if (FUSE) *tiles_started = ++started;          // the compress warps may take this tile's row block now
                 const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
                 const int m0 = t0.m0 + static_cast<int>(rank) * P_BM;
                 const int n0 = t0.n0 + static_cast<int>(rank) * (P_BN / 2);
@@ -260,7 +264,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int n_groups = (Kdim + 8 * cpr - 1) / (8 * cpr);
         auto walk = [&](auto vs) {
             vs.load(fz.v, fz.Dsub, lane);
-            for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+            int ti = 0;
+            for (int tile = pair; tile < num_tiles; tile += num_pairs, ++ti) {
+                if (!wait_for_tile(tiles_started, ti, abort_flag)) { failed = true; break; }
                 const PairTile t0 = pair_tile(tile, tiles_m, tiles_n);
                 const int r0 = t0.m0 + static_cast<int>(rank) * P_BM + cwi * 32;
                 if (r0 >= Mdim) continue;
