@@ -384,6 +384,42 @@ def run_ours(args):
                               "note": "the same step replayed from one captured graph (this rank's time)"}
 
     if not full:                                   # a parity-test configuration timed on request: the step only
+        # These configurations fit (partly) in L2, so the figure above is a WARM one: every step reads what the
+        # step before left in the cache.  The COLD figure rotates through enough copies of all buffers that a
+        # step finds none of its operands in L2 (the copies together hold more than twice the L2's 126 MB).
+        step_bytes = sum((N * (l["D"] + l["O"]) * 2 + l["O"] * l["D"] * 2) * 2 + N * l["M"] * 4 for l in L)
+        copies = int(min(16, max(2, -(-2 * 126e6 // step_bytes) + 1)))
+        sets = [L]
+        for _ in range(copies - 1):
+            # copies keep the row pitch of the originals (a plain clone would pack the padded rows)
+            sets.append([{k: (torch.empty_strided(v.shape, v.stride(), dtype=v.dtype, device=v.device).copy_(v)
+                              if isinstance(v, torch.Tensor) and v.is_cuda else v) for k, v in l.items()} for l in L])
+
+        def step_on(Ls):
+            for l in Ls:
+                vl.velora_linear_forward(l["X"], l["W"], l["v"], Y=l["Y"], Z=l["Z"], ws=ws)
+                vl.velora_linear_backward(l["dY"], l["W"], l["Z"], l["v"], dX=l["dX"], dW=l["dW"], ws=ws)
+
+        def time_steps(pick):
+            for Ls in sets:
+                step_on(Ls)
+            barrier()
+            cs, ce = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            cs.record()
+            for i in range(args.steps):
+                step_on(pick(i))
+            ce.record()
+            barrier()
+            return cs.elapsed_time(ce) / args.steps
+
+        warm_ms = time_steps(lambda i: sets[0])        # both without the per-layer events of the headline loop
+        cold_ms = time_steps(lambda i: sets[i % copies])
+        line["l2"] = {"warm_ms_per_step": warm_ms, "warm_tokens_per_s": N * world / (warm_ms * 1e-3),
+                      "cold_ms_per_step": cold_ms, "cold_tokens_per_s": N * world / (cold_ms * 1e-3),
+                      "copies_rotated": copies, "bytes_per_step": step_bytes,
+                      "note": "warm = one set of buffers step after step (partly L2-resident, like value / ms_per_step, which "
+                              "also carry three event records per layer); cold = the same step rotating through copies of "
+                              "every buffer so that nothing is found in L2"}
         if rank == 0:
             line["roofline"]["traffic"] = None         # the capture behind the ratio was taken on configuration 5
             print(json.dumps(line))

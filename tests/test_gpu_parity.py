@@ -240,6 +240,8 @@ FUSED_EDGE = [
     (130, 320, 1025, 256),   # sub-token spans four blocks, the last one has only one block of columns
     (513, 640, 1536, 128),   # sub-token spans two blocks
     (129, 2048, 1030, 1024), # longest sub-token
+    (260, 1536, 1100, 512),  # sub-token of 64 chunks: two loads per lane complete it
+    (140, 1000, 1026, 32),   # D a multiple of 8 only: the last 64-column block and the last sub-token are ragged
 ]
 
 
