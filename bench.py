@@ -746,6 +746,7 @@ def run_profile(args):
     torch.cuda.set_device(dev)
     cfg = vi.CONFIGS[CONFIG_INDEX]
     name = {"compress": "down", "reconstruct": "down", "init_v": "down", "weight_grad": "up",
+            "weight_grad_q": "q", "weight_grad_down": "down",
             "forward": "q", "input_grad": "q", "weight_grad_explicit": "q", "adapter_forward": "q",
             "adapter_weight_grad": "q", "adapter_input_grad": "q"}[args.profile]
     li = [l.name for l in cfg.layers].index(name)
@@ -777,7 +778,8 @@ def run_profile(args):
         Y = torch.empty((N, layer.O), dtype=torch.bfloat16, device=dev)
         dX = torch.empty_like(X)
         dW = torch.empty_like(W)
-        fn = {"weight_grad": lambda: vl.velora_weight_grad(dY, Z, v, layer.D, dW=dW, ws=ws),
+        wg = lambda: vl.velora_weight_grad(dY, Z, v, layer.D, dW=dW, ws=ws)
+        fn = {"weight_grad": wg, "weight_grad_q": wg, "weight_grad_down": wg,
               "weight_grad_explicit": lambda: vl.velora_weight_grad(dY, Z, v, layer.D, dW=dW, mode=vl.WG_EXPLICIT, ws=ws),
               "forward": lambda: vl.velora_linear_forward(X, W, v, Y=Y, Z=Z, ws=ws),
               "input_grad": lambda: vl.velora_linear_backward(dY, W, Z, v, dX=dX, need_dW=False, ws=ws)}[args.profile]
@@ -795,7 +797,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--profile", default=None,
-                    choices=["compress", "reconstruct", "init_v", "weight_grad", "weight_grad_explicit",
+                    choices=["compress", "reconstruct", "init_v", "weight_grad", "weight_grad_q", "weight_grad_down", "weight_grad_explicit",
                              "forward", "input_grad", "adapter_forward", "adapter_weight_grad", "adapter_input_grad"],
                     help="run four launches of one entry point on one layer (for ncu) and exit")
     ap.add_argument("--config", type=int, default=CONFIG_DEFAULT, choices=[2, 3, 4, 5],
