@@ -215,7 +215,11 @@ int launch_init_v_partials_rows(const void* X, int64_t N, int64_t D, int64_t ldx
     DeviceInfo di;
     const int rc = device_info(&di);
     if (rc != VELORA_OK) return rc;
-    const RowsPlan p = plan_rows(X, N, D, ldx, Dsub, di.sm_count, max_partials);
+    // Four CTAs of this kernel are resident per SM (its registers), so a grid of four per SM is one wave of CTAs
+    // that each walk a few rows; a larger grid would only add partial rows for the finalize kernel to add up.
+    int cap = di.sm_count * 4;
+    if (max_partials > 0 && cap > max_partials) cap = max_partials;
+    const RowsPlan p = plan_rows(X, N, D, ldx, Dsub, di.sm_count, cap);
     if (!p.ok) return VELORA_ERR_UNSUPPORTED;
     *num_partials = p.grid;
     return dispatch_rows<true, float>(p, X, N, D, ldx, nullptr, static_cast<float*>(nullptr), 0, partials, stream);
