@@ -126,8 +126,8 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t local_addr, uint32_t
 }
 
 // LPS, CH, WT describe the expansion (CLUSTER = true only): Dsub = 8 * LPS * CH, dW element type.
-template <bool CLUSTER, int LPS, int CH, typename WT>
-__global__ void __launch_bounds__(WG_THREADS, 2)
+template <bool CLUSTER, int LPS, int CH, typename WT, int NT = WG_THREADS>
+__global__ void __launch_bounds__(NT, NT == WG_THREADS ? 2 : 1)
 wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmZ, const WgArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -233,7 +233,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
             if (!failed) umma_commit(tfull);
             else *abort_flag = 1;
         }
-    } else {
+    } else if (warp < 6) {
         const int quarter = warp & 3;
         if (!mbar_wait_warp(tfull, 0u, abort_flag, 256)) {
             failed = true;
@@ -298,7 +298,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
         float* sp = reinterpret_cast<float*>(smem);
         if (a.splits > 1) {
             const int c4n = a.npad / 4;
-            for (int idx = threadIdx.x; idx < (r_end - r_begin) * c4n; idx += WG_THREADS) {
+            for (int idx = threadIdx.x; idx < (r_end - r_begin) * c4n; idx += NT) {
                 const int r = idx / c4n, c4 = idx - r * c4n;
                 const int off = (r_begin + r) * ldsp + c4 * 4;
                 const uint32_t laddr = base + static_cast<uint32_t>(off * 4);
@@ -315,7 +315,7 @@ wg_kernel(const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUten
             }
             __syncthreads();
         }
-        for (int trow = r_begin + warp; trow < r_end; trow += WG_THREADS / 32) {
+        for (int trow = r_begin + warp; trow < r_end; trow += NT / 32) {
             const int o = o0 + trow;
             if (o >= a.O) break;
             for (int m0 = 0; m0 < a.M; m0 += 32) {
@@ -372,6 +372,7 @@ struct WgPlan {
     bool ok;
     int M, npad, pitch, n_slabs, tmem_cols, kblocks, splits, kb_per_split, tiles_o, stages, tail_off;
     bool after_conversion;    // the launch follows z_to_bf16_kernel in the stream
+    bool fat;                 // one CTA of twelve warps per SM instead of two CTAs of six
     size_t zb_bytes, part_bytes, smem;
 };
 
@@ -398,11 +399,17 @@ WgPlan make_plan(int64_t N, int64_t D, int64_t O, int Dsub, int sm_count)
         return 1024 + ((body + 1023) / 1024) * 1024 + 256;
     };
     p.stages = WG_STAGES;
+    // One CTA per SM with twelve warps and half as many splits where the partial products are large (more than
+    // 64 sub-tokens) and there are few row blocks: the traffic of the cluster reduction halves, the ring is twice as
+    // deep and as many warps write dW (47 against 51 us on a 4096 x 11008 gradient with 172 sub-tokens).
+    p.fat = p.npad > 64 && static_cast<int64_t>(p.tiles_o) * 4 <= sm_count;
+    const bool fat = p.fat;
+    if (!fat)
     while (p.stages > 2 && 2 * (smem_for(p.stages) + 1024) > 228 * 1024) --p.stages;
-    if (2 * (smem_for(p.stages) + 1024) > 228 * 1024) p.stages = WG_STAGES;      // one CTA per SM either way
+    if (2 * (smem_for(p.stages) + 1024) > 228 * 1024) { p.stages = WG_STAGES; p.fat = true; }      // one CTA per SM either way: twelve warps
     p.smem = smem_for(p.stages);
     p.tail_off = static_cast<int>(p.smem - 1024 - 256);
-    const int64_t slots = static_cast<int64_t>(sm_count) * (2 * (p.smem + 1024) <= 228 * 1024 ? 2 : 1);
+    const int64_t slots = static_cast<int64_t>(sm_count) * ((!fat && 2 * (p.smem + 1024) <= 228 * 1024) ? 2 : 1);
     // Pick the split count that fills whole waves of SMs best; ties go to fewer splits (fewer partials).
     int best = 1;
     double best_eff = 0.0;
@@ -420,14 +427,14 @@ WgPlan make_plan(int64_t N, int64_t D, int64_t O, int Dsub, int sm_count)
     return p;
 }
 
-template <bool CLUSTER, int LPS, int CH, typename WT>
+template <bool CLUSTER, int LPS, int CH, typename WT, int NT = WG_THREADS>
 int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, const WgPlan& p, int smem_optin,
               cudaStream_t stream)
 {
     static DeviceOnce configured;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VELORA_ERR_CUDA;
-    auto kern = wg_kernel<CLUSTER, LPS, CH, WT>;
+    auto kern = wg_kernel<CLUSTER, LPS, CH, WT, NT>;
     if (!configured.get(dev)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
             return VELORA_ERR_CUDA;
@@ -435,7 +442,7 @@ int launch_wg(const CUtensorMap& tmY, const CUtensorMap& tmZ, const WgArgs& a, c
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(p.tiles_o), static_cast<unsigned>(p.splits), 1);
-    cfg.blockDim = dim3(WG_THREADS, 1, 1);
+    cfg.blockDim = dim3(NT, 1, 1);
     cfg.dynamicSmemBytes = p.smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -557,10 +564,16 @@ int launch_weight_grad_tc(const void* dY, int dy_dtype, int64_t N, int64_t O, in
         const int lps = L < 32 ? L : 32, ch = L / lps;
         rc = VELORA_ERR_CUDA;
 #define VELORA_WG_CASE(LPSV, CHV)                                                                             \
-        if (lps == LPSV && ch == CHV)                                                                         \
-            rc = dw_dtype == VELORA_BF16                                                                      \
-                     ? launch_wg<true, LPSV, CHV, __nv_bfloat16>(tmY, tmZ, a, plan, di.smem_optin, stream)       \
-                     : launch_wg<true, LPSV, CHV, float>(tmY, tmZ, a, plan, di.smem_optin, stream)
+        if (lps == LPSV && ch == CHV) {                                                                       \
+            if (plan.fat)                                                                                     \
+                rc = dw_dtype == VELORA_BF16                                                                  \
+                         ? launch_wg<true, LPSV, CHV, __nv_bfloat16, 2 * WG_THREADS>(tmY, tmZ, a, plan, di.smem_optin, stream) \
+                         : launch_wg<true, LPSV, CHV, float, 2 * WG_THREADS>(tmY, tmZ, a, plan, di.smem_optin, stream);        \
+            else                                                                                              \
+                rc = dw_dtype == VELORA_BF16                                                                  \
+                         ? launch_wg<true, LPSV, CHV, __nv_bfloat16>(tmY, tmZ, a, plan, di.smem_optin, stream)   \
+                         : launch_wg<true, LPSV, CHV, float>(tmY, tmZ, a, plan, di.smem_optin, stream);          \
+        }
         VELORA_WG_CASE(1, 1);
         VELORA_WG_CASE(2, 1);
         VELORA_WG_CASE(4, 1);
