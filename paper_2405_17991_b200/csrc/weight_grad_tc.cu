@@ -17,6 +17,9 @@
 //                      partials of its share of the 128 rows through distributed shared memory, in a
 //                      fixed order, and streams dW = P (x) v for those rows.  One launch, no partials in
 //                      global memory, every SM takes part in the write.
+//                      Two launch shapes: two CTAs of six warps per SM (ring of 2..4 stages), or, where the
+//                      partial products are large and the row blocks few, one CTA of twelve warps per SM with
+//                      half as many splits (half the reduction traffic, four stages, as many warps writing).
 //     CLUSTER = false  the partials go to the workspace and launch_expand_p sums and expands them
 //                      (shapes the cluster form does not take: Dsub not 8 * 2^k, unaligned dW rows).
 // Summing the partials in a fixed order keeps the result run-to-run identical.
