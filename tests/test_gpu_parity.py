@@ -198,6 +198,9 @@ EDGE = [
     (300, 260, 24, 2),     # four per chunk; D not a multiple of 8 (last chunk half real)
     (257, 104, 16, 1),     # eight per chunk
     (500, 99, 12, 4),      # ragged last sub-token (3 of 4) inside the last chunk
+    (700, 640, 300, 16),   # clustered weight gradient: three row blocks, the last one with 44 rows, 40 sub-tokens
+    (300, 520, 200, 8),    # ... 65 sub-tokens: the one-CTA-per-SM shape, two Zb slabs, five 64-token blocks to split
+    (1000, 1416, 130, 8),  # ... 177 sub-tokens (three slabs), a row block with two rows
 ]
 
 
